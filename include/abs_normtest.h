@@ -1,0 +1,183 @@
+/*
+ * abs_normtest.h -- C ABI of the norm-test + AdamW step for adaptive batch-size
+ * training ("Adaptive Batch Size Schedules for Distributed Training of Language
+ * Models with Data and Model Parallelism").
+ *
+ * One streaming pass over K worker (micro-batch) gradient buffers of a flat
+ * parameter vector of length d produces the averaged gradient, its squared norm,
+ * the between-worker variance sum, the paper's test statistic and next batch size,
+ * and (fused variant) the AdamW update that consumes the averaged gradient.
+ *
+ * Notation: the paper writes J for the number of workers; this API writes K.
+ *
+ * Conventions that hold for every launching entry point
+ *   - "device" pointers are memory of the CUDA device that is current on the calling
+ *     thread; "host" pointers are ordinary memory read during the call only.
+ *   - The caller owns every buffer.  The library allocates no device memory and
+ *     keeps no state between calls (abs_last_cuda_error aside).
+ *   - Work is enqueued on `stream` (a cudaStream_t; NULL = the legacy default
+ *     stream).  No call synchronises with the host; results are valid in stream order.
+ *   - Return value: ABS_OK, or a negative abs_status.  On a negative status nothing
+ *     was launched and no output was written.
+ *   - Results are deterministic: the same inputs give bit-identical outputs on every
+ *     call, independent of how the hardware schedules thread blocks.
+ */
+#ifndef ABS_NORMTEST_H_
+#define ABS_NORMTEST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void* abs_stream_t; /* a cudaStream_t */
+
+typedef enum { ABS_F32 = 0, ABS_BF16 = 1 } abs_dtype;
+
+typedef enum {
+  ABS_OK = 0,
+  ABS_ERR_NULL = -1,   /* a required pointer is NULL                                   */
+  ABS_ERR_RANGE = -2,  /* K, d, b, ld, step, eta, b_cur or a hyper-parameter is out of range */
+  ABS_ERR_SHARDS = -3, /* shard_offsets not non-decreasing, or ends are not 0 and d    */
+  ABS_ERR_ALIGN = -4,  /* a buffer is not aligned to its element size                  */
+  ABS_ERR_DTYPE = -5,  /* dtype is not an abs_dtype                                    */
+  ABS_ERR_CUDA = -6    /* a CUDA call failed; see abs_last_cuda_error()                */
+} abs_status;
+
+enum { ABS_MAX_WORKERS = 32, ABS_MAX_SHARDS = 128 };
+
+/* AdamW hyper-parameters (alpha, beta1, beta2, epsilon, lambda of Algorithm 1). */
+typedef struct {
+  float lr;
+  float beta1;
+  float beta2;
+  float eps;
+  float weight_decay;
+} abs_adamw_hparams;
+
+/*
+ * Layout of stats_out (device memory, doubles).  Header of ABS_STATS_HEADER doubles:
+ */
+enum {
+  ABS_STAT_N2 = 0,      /* ||gbar||^2, gbar as written/consumed in fp32                  */
+  ABS_STAT_S = 1,       /* sum_k ||g_k - gbar||^2   (per-sample form: sum over rows)     */
+  ABS_STAT_Q = 2,       /* sum_k ||g_k||^2          (diagnostic: S = Q - K*n2)           */
+  ABS_STAT_T = 3,       /* the statistic T                                               */
+  ABS_STAT_FLAGS = 4,   /* ABS_FLAG_* bits stored as a double                            */
+  ABS_STAT_NORM = 5,    /* K (worker form) or b-1 (per-sample form)                      */
+  ABS_STAT_NCHUNKS = 6, /* number of reduction chunks the call used                      */
+  ABS_STATS_HEADER = 8
+};
+/* then n_shards records of ABS_SHARD_STRIDE doubles {n2_s, S_s, Q_s, 0}, in shard order,
+ * then opaque scratch.  abs_stats_bytes() gives the total size.                        */
+enum { ABS_SHARD_STRIDE = 4 };
+
+enum {
+  ABS_FLAG_DEGENERATE = 1, /* ||gbar||^2 == 0                                           */
+  ABS_FLAG_NONFINITE = 2,  /* a sum is NaN or infinite; b_next = b_cur                  */
+  ABS_FLAG_VIOLATED = 4    /* T > b_cur: the test failed and b_next = ceil(T)           */
+};
+
+/* Bytes the caller must provide for stats_out of abs_norm_test / abs_normtest_adamw:
+ * header + shard records + chunk scratch.  Returns 0 on invalid arguments.  Host, pure. */
+size_t abs_stats_bytes(int64_t d, int n_shards);
+
+/* Bytes the caller must provide for stats_out of abs_persample_norm_test (b rows of d
+ * columns): header + one shard record + chunk scratch + the row-block work space.
+ * Returns 0 on invalid arguments.  Host, pure.                                          */
+size_t abs_persample_stats_bytes(int64_t b, int64_t d);
+
+/*
+ * DDP-Norm / FSDP-Norm test (Sec. 3.2-3.3; Algorithm 1 from "Compute the batch
+ * gradient" through the If/Else on T_k).
+ *   gbar[i] = (1/K) sum_k g_k[i]                      (mean over workers, fp32 out)
+ *   n2 = sum_i gbar[i]^2,  S = sum_k sum_i (g_k[i]-gbar[i])^2,  Q = sum_k sum_i g_k[i]^2
+ *   T = (S/K) / (eta^2 n2);   b_next = ceil(T) if T > b_cur else b_cur
+ * The same sums are also reported per shard of the flat vector (FSDP-Norm: each
+ * worker holds one parameter shard; Appendix A concatenates them); the totals are
+ * the shard records added in shard order.
+ *
+ *   grads          host array of K device pointers, each d elements of `dtype`,
+ *                  aligned to the element size (16-byte alignment is faster, not required)
+ *   K              1..ABS_MAX_WORKERS
+ *   d              >= 1
+ *   shard_offsets  host array of n_shards+1 non-decreasing offsets, [0]=0, [n_shards]=d;
+ *                  NULL = one shard (n_shards ignored)
+ *   n_shards       1..ABS_MAX_SHARDS
+ *   eta            finite, > 0 (the paper uses 0.05-0.275; values >= 1 are accepted)
+ *   b_cur          >= 1, the current global batch size
+ *   stats_out      device, abs_stats_bytes(d, n_shards) bytes, 16-byte aligned
+ *   gbar_out       device, d floats; must not alias any grads[k]
+ *   b_next_out     device, one int64
+ * Non-finite inputs are not an error: the flag is raised and b_next = b_cur.
+ */
+int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                  const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                  void* stats_out, float* gbar_out, int64_t* b_next_out, abs_stream_t stream);
+
+/*
+ * AdamW update (Algorithm 1, the five lines after the If/Else), in place, fp32:
+ *   m = beta1 m + (1-beta1) g;  v = beta2 v + (1-beta2) g^2
+ *   w = (1 - lr*wd) w - lr (m/(1-beta1^step)) / (sqrt(v/(1-beta2^step)) + eps)
+ *   params, m, v   device, d floats each, updated in place
+ *   gbar           device, d floats (e.g. gbar_out of abs_norm_test)
+ *   hparams        host; lr, eps, weight_decay finite and >= 0; beta1, beta2 in [0,1)
+ *   step           >= 1 (the k of Algorithm 1)
+ */
+int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t d,
+                   const abs_adamw_hparams* hparams, int64_t step, abs_stream_t stream);
+
+/*
+ * The fused step: abs_norm_test and abs_adamw_step in one pass, so gradients and
+ * optimizer state cross HBM once.  Arguments as above; gbar_out may be NULL (the mean
+ * then lives only in registers).  Legal because the update uses only the mean gradient
+ * and none of the test's results (Algorithm 1 lists the test first, with no data
+ * dependence between the two).
+ */
+int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                       const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                       void* stats_out, float* gbar_out, int64_t* b_next_out, float* params,
+                       float* m, float* v, const abs_adamw_hparams* hparams, int64_t step,
+                       abs_stream_t stream);
+
+/*
+ * Approximate norm test on per-sample gradients (Eq. 3, the Var definition before it,
+ * and the b_{k+1} display after it) -- the single-device form of the test.
+ *   G          device, row-major [b, ld]; row i = gradient of sample i; read once
+ *   b          >= 2 rows (also the current batch size), d >= 1 columns, ld >= d
+ *   dtype      ABS_F32 (ABS_BF16 is rejected with ABS_ERR_DTYPE)
+ *   gbar[c] = (1/b) sum_i G[i,c];  S = sum_i ||G[i,:]-gbar||^2;  ||Var||_1 = S/(b-1)
+ *   T = ||Var||_1 / (eta^2 ||gbar||^2);  b_next = ceil(T) if T > b else b
+ *   stats_out  device, abs_persample_stats_bytes(b, d) bytes, 16-byte aligned; header
+ *              as above with NORM = b-1 and one shard record
+ *   gbar_out   device, d floats;  b_next_out device, one int64
+ */
+int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs_dtype dtype,
+                            double eta, void* stats_out, float* gbar_out, int64_t* b_next_out,
+                            abs_stream_t stream);
+
+/*
+ * The decision alone, on the host, from sums already reduced (e.g. to re-decide for a
+ * different eta, or after combining per-rank sums in rank order).  Same expression
+ * order as the device code: T = (S/norm) / ((eta*eta)*n2).  Writes T and the ABS_FLAG_*
+ * bits when the pointers are non-NULL; returns b_next.  Pure.
+ */
+int64_t abs_decide(double S, double n2, double norm, double eta, int64_t b_cur, double* T_out,
+                   int* flags_out);
+
+/* Algorithm 1's rounding of a new batch size to the parallel layout:
+ * micro = ceil(b/(J*M)), mini = M*micro, returns J*mini.  J, M >= 1.  Returns -1 on
+ * invalid arguments.  Host, pure. */
+int64_t abs_round_batch(int64_t b_next, int64_t J, int64_t M);
+
+const char* abs_status_string(int status);
+
+/* The cudaError_t of the most recent ABS_ERR_CUDA on this thread (0 if none). */
+int abs_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ABS_NORMTEST_H_ */

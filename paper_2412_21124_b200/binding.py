@@ -1,0 +1,230 @@
+"""Thin ctypes binding of ``include/abs_normtest.h``.
+
+Argument marshalling only: every function here validates tensor types, collects raw
+device pointers and the current CUDA stream, and calls the C entry point of the same
+name.  All arithmetic of the path runs in the CUDA kernels of ``libabs_normtest.so``.
+There is no CPU fallback: if the library has not been built, the first call raises.
+"""
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+ABS_F32, ABS_BF16 = 0, 1
+ABS_OK = 0
+ABS_ERR_NULL, ABS_ERR_RANGE, ABS_ERR_SHARDS, ABS_ERR_ALIGN, ABS_ERR_DTYPE, ABS_ERR_CUDA = (
+    -1, -2, -3, -4, -5, -6)
+ABS_MAX_WORKERS, ABS_MAX_SHARDS = 32, 128
+(ABS_STAT_N2, ABS_STAT_S, ABS_STAT_Q, ABS_STAT_T, ABS_STAT_FLAGS, ABS_STAT_NORM,
+ ABS_STAT_NCHUNKS) = range(7)
+ABS_STATS_HEADER, ABS_SHARD_STRIDE = 8, 4
+ABS_FLAG_DEGENERATE, ABS_FLAG_NONFINITE, ABS_FLAG_VIOLATED = 1, 2, 4
+
+
+class abs_adamw_hparams(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float),
+                ("eps", ctypes.c_float), ("weight_decay", ctypes.c_float)]
+
+
+class AbsError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        msg = lib().abs_status_string(status).decode()
+        if status == ABS_ERR_CUDA:
+            msg += " [cudaError %d]" % lib().abs_last_cuda_error()
+        super().__init__("%s: %s (status %d)" % (where, msg, status))
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library.  Raises when it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(
+            "libabs_normtest.so is missing: build it with `python -m paper_2412_21124_b200.build` "
+            "(there is no CPU fallback)")
+    L = ctypes.CDLL(path)
+    i64, dbl, ptr, cint, sz = (ctypes.c_int64, ctypes.c_double, ctypes.c_void_p, ctypes.c_int,
+                               ctypes.c_size_t)
+    L.abs_stats_bytes.restype = sz
+    L.abs_stats_bytes.argtypes = [i64, cint]
+    L.abs_persample_stats_bytes.restype = sz
+    L.abs_persample_stats_bytes.argtypes = [i64, i64]
+    L.abs_norm_test.restype = cint
+    L.abs_norm_test.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64, ptr, ptr, ptr, ptr]
+    L.abs_adamw_step.restype = cint
+    L.abs_adamw_step.argtypes = [ptr, ptr, ptr, ptr, i64, ptr, i64, ptr]
+    L.abs_normtest_adamw.restype = cint
+    L.abs_normtest_adamw.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64, ptr, ptr, ptr,
+                                     ptr, ptr, ptr, ptr, i64, ptr]
+    L.abs_persample_norm_test.restype = cint
+    L.abs_persample_norm_test.argtypes = [ptr, i64, i64, i64, cint, dbl, ptr, ptr, ptr, ptr]
+    L.abs_decide.restype = i64
+    L.abs_decide.argtypes = [dbl, dbl, dbl, dbl, i64, ptr, ptr]
+    L.abs_round_batch.restype = i64
+    L.abs_round_batch.argtypes = [i64, i64, i64]
+    L.abs_status_string.restype = ctypes.c_char_p
+    L.abs_status_string.argtypes = [cint]
+    L.abs_last_cuda_error.restype = cint
+    L.abs_last_cuda_error.argtypes = []
+    _lib = L
+    return L
+
+
+# ------------------------------------------------------------------------- marshalling
+def _dtype_code(t):
+    if t.dtype == torch.float32:
+        return ABS_F32
+    if t.dtype == torch.bfloat16:
+        return ABS_BF16
+    raise TypeError("gradient buffers must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _check_f32_vec(t, d, name):
+    if t.dtype != torch.float32 or t.dim() != 1 or t.numel() != d or t.stride(0) != 1:
+        raise TypeError("%s must be a contiguous float32 vector of %d elements" % (name, d))
+    if not t.is_cuda:
+        raise TypeError("%s must live on a CUDA device" % name)
+
+
+def _stream(stream):
+    if stream is None:
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, torch.cuda.Stream):
+        return ctypes.c_void_p(stream.cuda_stream)
+    return ctypes.c_void_p(int(stream))
+
+
+def _grad_table(grads):
+    K = len(grads)
+    if K < 1:
+        raise ValueError("need at least one gradient buffer")
+    g0 = grads[0]
+    d, code = g0.numel(), _dtype_code(g0)
+    for g in grads:
+        if (not g.is_cuda or g.dtype != g0.dtype or g.dim() != 1 or g.numel() != d
+                or g.stride(0) != 1):
+            raise TypeError("gradient buffers must be contiguous CUDA vectors of one dtype/length")
+    table = (ctypes.c_void_p * K)(*[g.data_ptr() for g in grads])
+    return table, K, d, code
+
+
+def _offsets(shard_offsets):
+    if shard_offsets is None:
+        return None, 1
+    offs = (ctypes.c_int64 * len(shard_offsets))(*[int(o) for o in shard_offsets])
+    return offs, len(shard_offsets) - 1
+
+
+def _hparams(hp):
+    if isinstance(hp, abs_adamw_hparams):
+        return hp
+    return abs_adamw_hparams(float(hp["lr"]), float(hp["beta1"]), float(hp["beta2"]),
+                             float(hp["eps"]), float(hp["weight_decay"]))
+
+
+def abs_stats_bytes(d, n_shards=1):
+    return int(lib().abs_stats_bytes(int(d), int(n_shards)))
+
+
+def abs_persample_stats_bytes(b, d):
+    return int(lib().abs_persample_stats_bytes(int(b), int(d)))
+
+
+def alloc_stats(d, n_shards=1, device="cuda"):
+    """A stats_out buffer (float64 tensor) of the size abs_stats_bytes asks for."""
+    nbytes = abs_stats_bytes(d, n_shards)
+    if nbytes == 0:
+        raise ValueError("invalid (d, n_shards)")
+    return torch.empty(nbytes // 8, dtype=torch.float64, device=device)
+
+
+def alloc_persample_stats(b, d, device="cuda"):
+    nbytes = abs_persample_stats_bytes(b, d)
+    if nbytes == 0:
+        raise ValueError("invalid (b, d)")
+    return torch.empty(nbytes // 8, dtype=torch.float64, device=device)
+
+
+# ------------------------------------------------------------------------- entry points
+def abs_norm_test(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offsets=None,
+                  stream=None):
+    table, K, d, code = _grad_table(grads)
+    offs, n_shards = _offsets(shard_offsets)
+    _check_f32_vec(gbar_out, d, "gbar_out")
+    rc = lib().abs_norm_test(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
+                             stats_out.data_ptr(), gbar_out.data_ptr(), b_next_out.data_ptr(),
+                             _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_norm_test")
+
+
+def abs_adamw_step(params, gbar, m, v, hparams, step, stream=None):
+    d = params.numel()
+    for t, name in ((params, "params"), (gbar, "gbar"), (m, "m"), (v, "v")):
+        _check_f32_vec(t, d, name)
+    hp = _hparams(hparams)
+    rc = lib().abs_adamw_step(params.data_ptr(), gbar.data_ptr(), m.data_ptr(), v.data_ptr(), d,
+                              ctypes.byref(hp), int(step), _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_adamw_step")
+
+
+def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v, hparams,
+                       step, shard_offsets=None, stream=None):
+    table, K, d, code = _grad_table(grads)
+    offs, n_shards = _offsets(shard_offsets)
+    for t, name in ((params, "params"), (m, "m"), (v, "v")):
+        _check_f32_vec(t, d, name)
+    if gbar_out is not None:
+        _check_f32_vec(gbar_out, d, "gbar_out")
+    hp = _hparams(hparams)
+    rc = lib().abs_normtest_adamw(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
+                                  stats_out.data_ptr(),
+                                  gbar_out.data_ptr() if gbar_out is not None else None,
+                                  b_next_out.data_ptr(), params.data_ptr(), m.data_ptr(),
+                                  v.data_ptr(), ctypes.byref(hp), int(step), _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_normtest_adamw")
+
+
+def abs_persample_norm_test(G, eta, stats_out, gbar_out, b_next_out, stream=None):
+    if G.dim() != 2 or G.stride(1) != 1 or not G.is_cuda:
+        raise TypeError("G must be a CUDA matrix [b, d] with unit column stride")
+    b, d, ld = G.shape[0], G.shape[1], G.stride(0)
+    _check_f32_vec(gbar_out, d, "gbar_out")
+    rc = lib().abs_persample_norm_test(G.data_ptr(), b, d, ld, _dtype_code(G), float(eta),
+                                       stats_out.data_ptr(), gbar_out.data_ptr(),
+                                       b_next_out.data_ptr(), _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_persample_norm_test")
+
+
+def abs_decide(S, n2, norm, eta, b_cur):
+    """Host-side decision; returns (b_next, T, flags)."""
+    T, flags = ctypes.c_double(0.0), ctypes.c_int(0)
+    b_next = lib().abs_decide(float(S), float(n2), float(norm), float(eta), int(b_cur),
+                              ctypes.byref(T), ctypes.byref(flags))
+    return int(b_next), T.value, flags.value
+
+
+def abs_round_batch(b_next, J, M):
+    return int(lib().abs_round_batch(int(b_next), int(J), int(M)))
+
+
+def read_stats(stats_out, n_shards=1):
+    """Copies the header and shard records to the host (synchronises) and names them."""
+    n = ABS_STATS_HEADER + n_shards * ABS_SHARD_STRIDE
+    h = stats_out[:n].cpu().tolist()
+    shards = [tuple(h[ABS_STATS_HEADER + s * ABS_SHARD_STRIDE + j] for j in range(3))
+              for s in range(n_shards)]
+    return {"n2": h[ABS_STAT_N2], "S": h[ABS_STAT_S], "Q": h[ABS_STAT_Q], "T": h[ABS_STAT_T],
+            "flags": int(h[ABS_STAT_FLAGS]), "norm": h[ABS_STAT_NORM],
+            "n_chunks": int(h[ABS_STAT_NCHUNKS]), "shards": shards}

@@ -1,0 +1,363 @@
+// C ABI of the norm-test + AdamW library: argument validation, launch configuration and
+// the host-side helpers.  Every step of the path runs in the kernels; this file only
+// checks, sizes and launches.
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+#include "abs_device.cuh"
+#include "normtest_stream.cuh"
+#include "persample.cuh"
+
+using namespace absnt;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = static_cast<int>(e);
+  return ABS_ERR_CUDA;
+}
+
+// Elements per reduction chunk.  A function of d alone, so that the summation tree --
+// and with it every output bit -- depends only on the problem, not on the launch.
+int chunk_elems_for(int64_t d) { return d >= (int64_t{1} << 23) ? 16384 : 4096; }
+
+bool finite_nonneg(float x) { return std::isfinite(x) && x >= 0.f; }
+
+int check_hparams(const abs_adamw_hparams* h, int64_t step) {
+  if (!h) return ABS_ERR_NULL;
+  if (step < 1) return ABS_ERR_RANGE;
+  if (!finite_nonneg(h->lr) || !finite_nonneg(h->eps) || !finite_nonneg(h->weight_decay))
+    return ABS_ERR_RANGE;
+  if (!(h->beta1 >= 0.f && h->beta1 < 1.f) || !(h->beta2 >= 0.f && h->beta2 < 1.f))
+    return ABS_ERR_RANGE;
+  return ABS_OK;
+}
+
+AdamScalars make_adam(const abs_adamw_hparams* h, int64_t step) {
+  AdamScalars a;
+  const double b1 = h->beta1, b2 = h->beta2;
+  a.beta1 = h->beta1;
+  a.omb1 = static_cast<float>(1.0 - b1);
+  a.beta2 = h->beta2;
+  a.omb2 = static_cast<float>(1.0 - b2);
+  a.inv_bc1 = static_cast<float>(1.0 / (1.0 - std::pow(b1, static_cast<double>(step))));
+  a.inv_bc2 = static_cast<float>(1.0 / (1.0 - std::pow(b2, static_cast<double>(step))));
+  a.lr = h->lr;
+  a.eps = h->eps;
+  a.decay =
+      static_cast<float>(1.0 - static_cast<double>(h->lr) * static_cast<double>(h->weight_decay));
+  return a;
+}
+
+bool misaligned(const void* p, size_t a) {
+  return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
+}
+
+struct Layout {
+  int n_shards;
+  int n_chunks;
+  int chunk_elems;
+  int64_t shard_off[ABS_MAX_SHARDS + 1];
+  int32_t chunk_prefix[ABS_MAX_SHARDS + 1];
+};
+
+// Validates the shard table and cuts the shards into chunks.
+int make_layout(int64_t d, const int64_t* shard_offsets, int n_shards, Layout* L) {
+  if (!shard_offsets) n_shards = 1;
+  if (n_shards < 1 || n_shards > ABS_MAX_SHARDS) return ABS_ERR_RANGE;
+  L->n_shards = n_shards;
+  L->chunk_elems = chunk_elems_for(d);
+  if (!shard_offsets) {
+    L->shard_off[0] = 0;
+    L->shard_off[1] = d;
+  } else {
+    if (shard_offsets[0] != 0 || shard_offsets[n_shards] != d) return ABS_ERR_SHARDS;
+    for (int s = 0; s < n_shards; ++s)
+      if (shard_offsets[s + 1] < shard_offsets[s]) return ABS_ERR_SHARDS;
+    std::memcpy(L->shard_off, shard_offsets, sizeof(int64_t) * (n_shards + 1));
+  }
+  int64_t chunks = 0;
+  for (int s = 0; s < n_shards; ++s) {
+    L->chunk_prefix[s] = static_cast<int32_t>(chunks);
+    chunks += (L->shard_off[s + 1] - L->shard_off[s] + L->chunk_elems - 1) / L->chunk_elems;
+    if (chunks > INT32_MAX) return ABS_ERR_RANGE;
+  }
+  L->chunk_prefix[n_shards] = static_cast<int32_t>(chunks);
+  L->n_chunks = static_cast<int>(chunks);
+  return ABS_OK;
+}
+
+template <typename GT, bool ADAM>
+cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
+  const int grid = prm.n_chunks;
+  const int K = prm.K;
+#define ABS_LAUNCH(KB, EXACT) \
+  normtest_stream_kernel<GT, KB, EXACT, ADAM><<<grid, kThreads, 0, st>>>(prm)
+  switch (K) {
+    case 1: ABS_LAUNCH(1, true); break;
+    case 2: ABS_LAUNCH(2, true); break;
+    case 3: ABS_LAUNCH(3, true); break;
+    case 4: ABS_LAUNCH(4, true); break;
+    case 8: ABS_LAUNCH(8, true); break;
+    case 16: ABS_LAUNCH(16, true); break;
+    case 32: ABS_LAUNCH(32, true); break;
+    default:
+      if (K < 8) ABS_LAUNCH(8, false);
+      else if (K < 16) ABS_LAUNCH(16, false);
+      else ABS_LAUNCH(32, false);
+  }
+#undef ABS_LAUNCH
+  return cudaGetLastError();
+}
+
+int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                  const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                  void* stats_out, float* gbar_out, int64_t* b_next_out, float* params, float* m,
+                  float* v, const abs_adamw_hparams* hparams, int64_t step, bool fused,
+                  abs_stream_t stream) {
+  if (!grads || !stats_out || !b_next_out) return ABS_ERR_NULL;
+  if (!fused && !gbar_out) return ABS_ERR_NULL;
+  if (fused && (!params || !m || !v)) return ABS_ERR_NULL;
+  if (dtype != ABS_F32 && dtype != ABS_BF16) return ABS_ERR_DTYPE;
+  if (K < 1 || K > ABS_MAX_WORKERS || d < 1 || b_cur < 1) return ABS_ERR_RANGE;
+  if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
+  if (fused) {
+    const int rc = check_hparams(hparams, step);
+    if (rc != ABS_OK) return rc;
+  }
+  const size_t esz = (dtype == ABS_F32) ? 4 : 2;
+  for (int k = 0; k < K; ++k) {
+    if (!grads[k]) return ABS_ERR_NULL;
+    if (misaligned(grads[k], esz)) return ABS_ERR_ALIGN;
+  }
+  if (misaligned(stats_out, 16) || misaligned(b_next_out, 8)) return ABS_ERR_ALIGN;
+  if (gbar_out && misaligned(gbar_out, 4)) return ABS_ERR_ALIGN;
+  if (fused && (misaligned(params, 4) || misaligned(m, 4) || misaligned(v, 4)))
+    return ABS_ERR_ALIGN;
+
+  Layout L;
+  const int rc = make_layout(d, shard_offsets, n_shards, &L);
+  if (rc != ABS_OK) return rc;
+
+  double* stats = static_cast<double*>(stats_out);
+  double* chunk_out =
+      stats + ABS_STATS_HEADER + static_cast<size_t>(L.n_shards) * ABS_SHARD_STRIDE;
+
+  StreamParams prm;
+  std::memset(&prm, 0, sizeof prm);
+  for (int k = 0; k < K; ++k) prm.grads[k] = grads[k];
+  std::memcpy(prm.shard_off, L.shard_off, sizeof(int64_t) * (L.n_shards + 1));
+  std::memcpy(prm.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
+  prm.d = d;
+  prm.K = K;
+  prm.n_shards = L.n_shards;
+  prm.n_chunks = L.n_chunks;
+  prm.chunk_elems = L.chunk_elems;
+  prm.inv_K = 1.0 / static_cast<double>(K);
+  prm.gbar = gbar_out;
+  prm.p = params;
+  prm.m = m;
+  prm.v = v;
+  prm.chunk_out = chunk_out;
+  if (fused) prm.adam = make_adam(hparams, step);
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  if (dtype == ABS_F32)
+    e = fused ? launch_stream<F32, true>(prm, st) : launch_stream<F32, false>(prm, st);
+  else
+    e = fused ? launch_stream<BF16, true>(prm, st) : launch_stream<BF16, false>(prm, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+
+  FinalizeParams fp;
+  std::memset(&fp, 0, sizeof fp);
+  fp.chunk_in = chunk_out;
+  std::memcpy(fp.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
+  fp.n_shards = L.n_shards;
+  fp.n_chunks = L.n_chunks;
+  fp.stats = stats;
+  fp.b_next = b_next_out;
+  fp.eta = eta;
+  fp.norm = static_cast<double>(K);
+  fp.b_cur = b_cur;
+  finalize_kernel<<<1, kFinalizeThreads, 0, st>>>(fp);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return ABS_OK;
+}
+
+int persample_rows_per_block(int64_t b) { return b >= 2048 ? 128 : (b >= 512 ? 64 : 32); }
+
+}  // namespace
+
+extern "C" {
+
+size_t abs_stats_bytes(int64_t d, int n_shards) {
+  if (d < 1 || n_shards < 1 || n_shards > ABS_MAX_SHARDS) return 0;
+  const int ce = chunk_elems_for(d);
+  const int64_t max_chunks = (d + ce - 1) / ce + n_shards;
+  return sizeof(double) * (ABS_STATS_HEADER + static_cast<size_t>(n_shards) * ABS_SHARD_STRIDE +
+                           static_cast<size_t>(max_chunks) * 4);
+}
+
+size_t abs_persample_stats_bytes(int64_t b, int64_t d) {
+  if (b < 2 || d < 1) return 0;
+  const int rpb = persample_rows_per_block(b);
+  const int64_t nrb = (b + rpb - 1) / rpb;
+  const int64_t n_chunks = (d + kThreads - 1) / kThreads;
+  return sizeof(double) *
+         (ABS_STATS_HEADER + ABS_SHARD_STRIDE + static_cast<size_t>(n_chunks) * 4 +
+          3 * static_cast<size_t>(nrb) * static_cast<size_t>(d));
+}
+
+int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                  const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                  void* stats_out, float* gbar_out, int64_t* b_next_out, abs_stream_t stream) {
+  return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
+                       gbar_out, b_next_out, nullptr, nullptr, nullptr, nullptr, 0, false, stream);
+}
+
+int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                       const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                       void* stats_out, float* gbar_out, int64_t* b_next_out, float* params,
+                       float* m, float* v, const abs_adamw_hparams* hparams, int64_t step,
+                       abs_stream_t stream) {
+  return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
+                       gbar_out, b_next_out, params, m, v, hparams, step, true, stream);
+}
+
+int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t d,
+                   const abs_adamw_hparams* hparams, int64_t step, abs_stream_t stream) {
+  if (!params || !gbar || !m || !v) return ABS_ERR_NULL;
+  if (d < 1) return ABS_ERR_RANGE;
+  const int rc = check_hparams(hparams, step);
+  if (rc != ABS_OK) return rc;
+  if (misaligned(params, 4) || misaligned(gbar, 4) || misaligned(m, 4) || misaligned(v, 4))
+    return ABS_ERR_ALIGN;
+  const AdamScalars a = make_adam(hparams, step);
+  const bool vec = !(misaligned(params, 16) || misaligned(gbar, 16) || misaligned(m, 16) ||
+                     misaligned(v, 16));
+  const int64_t work = vec ? (d + 3) / 4 : d;
+  int64_t blocks = (work + kThreads - 1) / kThreads;
+  const int64_t cap = 148 * 16;
+  if (blocks > cap) blocks = cap;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (vec)
+    adamw_kernel<true><<<static_cast<int>(blocks), kThreads, 0, st>>>(params, gbar, m, v, d, a);
+  else
+    adamw_kernel<false><<<static_cast<int>(blocks), kThreads, 0, st>>>(params, gbar, m, v, d, a);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return ABS_OK;
+}
+
+int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs_dtype dtype,
+                            double eta, void* stats_out, float* gbar_out, int64_t* b_next_out,
+                            abs_stream_t stream) {
+  if (!G || !stats_out || !gbar_out || !b_next_out) return ABS_ERR_NULL;
+  if (dtype != ABS_F32) return ABS_ERR_DTYPE;
+  if (b < 2 || d < 1 || ld < d) return ABS_ERR_RANGE;
+  if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
+  if (misaligned(G, 4) || misaligned(gbar_out, 4) || misaligned(stats_out, 16) ||
+      misaligned(b_next_out, 8))
+    return ABS_ERR_ALIGN;
+  const int64_t n_chunks64 = (d + kThreads - 1) / kThreads;
+  const int rpb = persample_rows_per_block(b);
+  const int64_t nrb = (b + rpb - 1) / rpb;
+  if (n_chunks64 > INT32_MAX || nrb > 65535) return ABS_ERR_RANGE;
+
+  double* stats = static_cast<double*>(stats_out);
+  PersampleParams prm;
+  std::memset(&prm, 0, sizeof prm);
+  prm.G = static_cast<const float*>(G);
+  prm.b = b;
+  prm.d = d;
+  prm.ld = ld;
+  prm.rows_per_block = rpb;
+  prm.n_row_blocks = static_cast<int>(nrb);
+  prm.chunk_out = stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE;
+  prm.ws_mean = prm.chunk_out + n_chunks64 * 4;
+  prm.ws_m2 = prm.ws_mean + nrb * d;
+  prm.ws_q = prm.ws_m2 + nrb * d;
+  prm.gbar = gbar_out;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool vec = !misaligned(G, 16) && (ld % 4 == 0);
+  if (vec) {
+    const int64_t cols = (d + 3) / 4;
+    dim3 grid(static_cast<unsigned>((cols + kThreads - 1) / kThreads),
+              static_cast<unsigned>(nrb));
+    persample_partial_kernel<4><<<grid, kThreads, 0, st>>>(prm);
+  } else {
+    dim3 grid(static_cast<unsigned>(n_chunks64), static_cast<unsigned>(nrb));
+    persample_partial_kernel<1><<<grid, kThreads, 0, st>>>(prm);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  persample_merge_kernel<<<static_cast<int>(n_chunks64), kThreads, 0, st>>>(prm);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+
+  FinalizeParams fp;
+  std::memset(&fp, 0, sizeof fp);
+  fp.chunk_in = prm.chunk_out;
+  fp.chunk_prefix[0] = 0;
+  fp.chunk_prefix[1] = static_cast<int32_t>(n_chunks64);
+  fp.n_shards = 1;
+  fp.n_chunks = static_cast<int>(n_chunks64);
+  fp.stats = stats;
+  fp.b_next = b_next_out;
+  fp.eta = eta;
+  fp.norm = static_cast<double>(b - 1);
+  fp.b_cur = b;
+  finalize_kernel<<<1, kFinalizeThreads, 0, st>>>(fp);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return ABS_OK;
+}
+
+int64_t abs_decide(double S, double n2, double norm, double eta, int64_t b_cur, double* T_out,
+                   int* flags_out) {
+  int flags = 0;
+  const double T = (S / norm) / ((eta * eta) * n2);
+  int64_t b_next = b_cur;
+  if (!std::isfinite(S) || !std::isfinite(n2)) {
+    flags |= ABS_FLAG_NONFINITE;
+  } else {
+    if (n2 == 0.0) flags |= ABS_FLAG_DEGENERATE;
+    if (T > static_cast<double>(b_cur)) {
+      flags |= ABS_FLAG_VIOLATED;
+      b_next = (T >= 4611686018427387904.0) ? INT64_MAX : static_cast<int64_t>(std::ceil(T));
+    }
+  }
+  if (T_out) *T_out = T;
+  if (flags_out) *flags_out = flags;
+  return b_next;
+}
+
+int64_t abs_round_batch(int64_t b_next, int64_t J, int64_t M) {
+  if (b_next < 1 || J < 1 || M < 1) return -1;
+  const int64_t jm = J * M;
+  const int64_t micro = (b_next + jm - 1) / jm;
+  return J * (M * micro);
+}
+
+const char* abs_status_string(int status) {
+  switch (status) {
+    case ABS_OK: return "ok";
+    case ABS_ERR_NULL: return "a required pointer is NULL";
+    case ABS_ERR_RANGE: return "an argument is out of range";
+    case ABS_ERR_SHARDS: return "shard offsets are not a non-decreasing cover of [0, d]";
+    case ABS_ERR_ALIGN: return "a buffer is not aligned to its element size";
+    case ABS_ERR_DTYPE: return "unsupported dtype";
+    case ABS_ERR_CUDA: return "a CUDA call failed (see abs_last_cuda_error)";
+    default: return "unknown status";
+  }
+}
+
+int abs_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

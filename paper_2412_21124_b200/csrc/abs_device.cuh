@@ -1,0 +1,161 @@
+// Device-side building blocks shared by the kernels of the norm-test + AdamW library:
+// kernel parameter blocks, streaming 128-bit loads/stores, bf16 unpacking, the AdamW
+// element update and the fixed-shape fp64 block reduction.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/abs_normtest.h"
+
+namespace absnt {
+
+constexpr int kThreads = 256;  // threads per CTA of the streaming kernels
+constexpr int kWarps = kThreads / 32;
+
+// AdamW scalars (Algorithm 1, AdamW lines), prepared on the host in double.
+struct AdamScalars {
+  float beta1, omb1;      // beta1, 1-beta1
+  float beta2, omb2;      // beta2, 1-beta2
+  float inv_bc1, inv_bc2; // 1/(1-beta1^step), 1/(1-beta2^step)
+  float lr, eps, decay;   // alpha, epsilon, 1-alpha*lambda
+};
+
+// Parameter block of the streaming norm-test kernels, passed by value.
+struct StreamParams {
+  const void* grads[ABS_MAX_WORKERS];
+  int64_t shard_off[ABS_MAX_SHARDS + 1];    // element offsets of the shards
+  int32_t chunk_prefix[ABS_MAX_SHARDS + 1]; // first chunk index of each shard
+  int64_t d;
+  int K;
+  int n_shards;
+  int n_chunks;
+  int chunk_elems; // elements per reduction chunk (a multiple of kThreads*8)
+  double inv_K;
+  float* gbar; // may be null
+  float* p;    // fused AdamW only
+  float* m;
+  float* v;
+  double* chunk_out; // 4 doubles per chunk: n2, S, Q, 0
+  AdamScalars adam;
+};
+
+struct FinalizeParams {
+  const double* chunk_in;
+  int32_t chunk_prefix[ABS_MAX_SHARDS + 1];
+  int n_shards;
+  int n_chunks;
+  double* stats; // header + shard records
+  int64_t* b_next;
+  double eta, norm;
+  int64_t b_cur;
+};
+
+// ---- streaming memory access --------------------------------------------------------
+// Gradients are read exactly once and never written: non-coherent path, no L1 allocation.
+__device__ __forceinline__ uint4 ld_once_16(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+// Optimizer state is read once and then overwritten by the same thread.
+__device__ __forceinline__ float4 ld_state_16(const float* p) {
+  return __ldcs(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ void st_stream_16(float* p, float4 x) {
+  __stcs(reinterpret_cast<float4*>(p), x);
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Element types of the gradient buffers.
+struct F32 {
+  static constexpr int kVec = 4; // elements per 16 bytes
+  using scalar = float;
+  static __device__ __forceinline__ float elem(const uint4& r, int e) {
+    return __uint_as_float(e == 0 ? r.x : e == 1 ? r.y : e == 2 ? r.z : r.w);
+  }
+  static __device__ __forceinline__ float load1(const void* base, int64_t i) {
+    return __ldg(reinterpret_cast<const float*>(base) + i);
+  }
+};
+struct BF16 {
+  static constexpr int kVec = 8;
+  using scalar = uint16_t;
+  static __device__ __forceinline__ float elem(const uint4& r, int e) {
+    const uint32_t w = (e >> 1) == 0 ? r.x : (e >> 1) == 1 ? r.y : (e >> 1) == 2 ? r.z : r.w;
+    return (e & 1) ? bf16_hi(w) : bf16_lo(w);
+  }
+  static __device__ __forceinline__ float load1(const void* base, int64_t i) {
+    return __uint_as_float(
+        static_cast<uint32_t>(__ldg(reinterpret_cast<const uint16_t*>(base) + i)) << 16);
+  }
+};
+
+// One AdamW coordinate (Algorithm 1: m_k, v_k, the two hats, w_{k+1}).
+__device__ __forceinline__ void adamw_elem(const AdamScalars& a, float g, float& w, float& m,
+                                           float& v) {
+  m = fmaf(a.beta1, m, a.omb1 * g);
+  v = fmaf(a.beta2, v, a.omb2 * (g * g));
+  const float mhat = m * a.inv_bc1;
+  const float vhat = v * a.inv_bc2;
+  const float denom = sqrtf(vhat) + a.eps;
+  w = fmaf(a.decay, w, -(a.lr * (mhat / denom)));
+}
+
+// Fixed-shape reduction of three doubles over a CTA of NW warps.  Every call adds the
+// same operands in the same order, so the result is independent of scheduling.
+// Result valid in thread 0.  `sm` holds NW*3 doubles.
+template <int NW>
+__device__ __forceinline__ void block_reduce3(double& a, double& b, double& c, double* sm) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    a += __shfl_down_sync(0xffffffffu, a, off);
+    b += __shfl_down_sync(0xffffffffu, b, off);
+    c += __shfl_down_sync(0xffffffffu, c, off);
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) {
+    sm[warp * 3 + 0] = a;
+    sm[warp * 3 + 1] = b;
+    sm[warp * 3 + 2] = c;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double ra = sm[0], rb = sm[1], rc = sm[2];
+#pragma unroll
+    for (int w = 1; w < NW; ++w) {
+      ra += sm[w * 3 + 0];
+      rb += sm[w * 3 + 1];
+      rc += sm[w * 3 + 2];
+    }
+    a = ra;
+    b = rb;
+    c = rc;
+  }
+  __syncthreads();
+}
+
+// The decision, device side (same expression order as the host's abs_decide).
+__device__ __forceinline__ int64_t decide_device(double S, double n2, double norm, double eta,
+                                                 int64_t b_cur, double* T_out, int* flags_out) {
+  int flags = 0;
+  const double T = (S / norm) / ((eta * eta) * n2);
+  int64_t b_next = b_cur;
+  if (!isfinite(S) || !isfinite(n2)) {
+    flags |= ABS_FLAG_NONFINITE;
+  } else {
+    if (n2 == 0.0) flags |= ABS_FLAG_DEGENERATE;
+    if (T > static_cast<double>(b_cur)) {
+      flags |= ABS_FLAG_VIOLATED;
+      b_next = (T >= 4611686018427387904.0) ? INT64_MAX : static_cast<int64_t>(ceil(T));
+    }
+  }
+  *T_out = T;
+  *flags_out = flags;
+  return b_next;
+}
+
+}  // namespace absnt

@@ -1,0 +1,185 @@
+// Per-sample form of the norm test (Eq. 3 with the Var definition before it): column
+// mean and column sum of squared deviations of a row-major [b, ld] matrix whose rows
+// are per-sample gradients, reading the matrix once.
+//
+// Pass 1 (2-D grid: column block x row block): a thread owns VC adjacent columns and
+// walks its row block in groups of kGroup rows held in registers.  Per group and
+// column it forms the group mean (fp64 sum) and the within-group squared deviations
+// (fp32), and merges them into running {mean, M2} with the pairwise update
+//     delta = mu_g - mean;  mean += delta*n_g/(n+n_g);  M2 += M2_g + delta^2*n*n_g/(n+n_g)
+// (law of total variance).  It writes {mean, M2, Q} per (row block, column).
+// Pass 2 (one thread per column): merges the row blocks in index order with the same
+// update, writes gbar, and reduces {gbar^2, M2, Q} over 256-column chunks for the
+// shared finalize kernel.
+// Also here: the stand-alone AdamW kernel.
+#pragma once
+#include "abs_device.cuh"
+
+namespace absnt {
+
+constexpr int kGroup = 16; // rows held in registers at a time
+
+struct PersampleParams {
+  const float* G;
+  int64_t b, d, ld;
+  int rows_per_block;
+  int n_row_blocks;
+  double* ws_mean; // [n_row_blocks][d]
+  double* ws_m2;
+  double* ws_q;
+  float* gbar;
+  double* chunk_out; // 4 doubles per 256-column chunk
+};
+
+template <int VC>
+__global__ void __launch_bounds__(kThreads)
+    persample_partial_kernel(const __grid_constant__ PersampleParams prm) {
+  const int64_t c0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) * VC;
+  if (c0 >= prm.d) return;
+  const int64_t r0 = static_cast<int64_t>(blockIdx.y) * prm.rows_per_block;
+  const int64_t r1 = (r0 + prm.rows_per_block < prm.b) ? r0 + prm.rows_per_block : prm.b;
+  const bool full_cols = (c0 + VC <= prm.d);
+
+  double mean[VC], m2[VC], qq[VC];
+#pragma unroll
+  for (int i = 0; i < VC; ++i) mean[i] = m2[i] = qq[i] = 0.0;
+  int n = 0;
+
+  for (int64_t r = r0; r < r1; r += kGroup) {
+    const int ng = (r1 - r < kGroup) ? static_cast<int>(r1 - r) : kGroup;
+    float x[kGroup][VC];
+#pragma unroll
+    for (int j = 0; j < kGroup; ++j) {
+      const float* row = prm.G + (r + j) * prm.ld + c0;
+      if (j < ng) {
+        if (VC == 4 && full_cols) {
+          const uint4 t = ld_once_16(row);
+          x[j][0] = __uint_as_float(t.x);
+          x[j][1 % VC] = __uint_as_float(t.y);
+          x[j][2 % VC] = __uint_as_float(t.z);
+          x[j][3 % VC] = __uint_as_float(t.w);
+        } else {
+#pragma unroll
+          for (int i = 0; i < VC; ++i) x[j][i] = (c0 + i < prm.d) ? __ldg(row + i) : 0.f;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < VC; ++i) x[j][i] = 0.f;
+      }
+    }
+    const double inv_ng = 1.0 / static_cast<double>(ng);
+    const double nn = static_cast<double>(n + ng);
+    const double w_mean = static_cast<double>(ng) / nn;
+    const double w_m2 = static_cast<double>(n) * w_mean;
+#pragma unroll
+    for (int i = 0; i < VC; ++i) {
+      double s = 0.0;
+#pragma unroll
+      for (int j = 0; j < kGroup; ++j) s += static_cast<double>(x[j][i]); // absent rows are 0
+      const double mu = s * inv_ng;
+      const float muf = static_cast<float>(mu);
+      float dev2 = 0.f, sq = 0.f;
+#pragma unroll
+      for (int j = 0; j < kGroup; ++j) {
+        if (j < ng) {
+          const float dv = x[j][i] - muf;
+          dev2 = fmaf(dv, dv, dev2);
+          sq = fmaf(x[j][i], x[j][i], sq);
+        }
+      }
+      const double delta = mu - mean[i];
+      mean[i] += delta * w_mean;
+      m2[i] += static_cast<double>(dev2) + delta * delta * w_m2;
+      qq[i] += static_cast<double>(sq);
+    }
+    n += ng;
+  }
+  const int64_t o = static_cast<int64_t>(blockIdx.y) * prm.d + c0;
+#pragma unroll
+  for (int i = 0; i < VC; ++i) {
+    if (c0 + i < prm.d) {
+      prm.ws_mean[o + i] = mean[i];
+      prm.ws_m2[o + i] = m2[i];
+      prm.ws_q[o + i] = qq[i];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+    persample_merge_kernel(const __grid_constant__ PersampleParams prm) {
+  __shared__ double red[kWarps * 3];
+  const int64_t c = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  double a = 0.0, s = 0.0, q = 0.0;
+  if (c < prm.d) {
+    double mean = 0.0, m2 = 0.0;
+    int64_t n = 0;
+    for (int rb = 0; rb < prm.n_row_blocks; ++rb) {
+      const int64_t r0 = static_cast<int64_t>(rb) * prm.rows_per_block;
+      const int64_t nb = (r0 + prm.rows_per_block < prm.b) ? prm.rows_per_block : prm.b - r0;
+      const double mu = prm.ws_mean[static_cast<int64_t>(rb) * prm.d + c];
+      const double nn = static_cast<double>(n + nb);
+      const double w_mean = static_cast<double>(nb) / nn;
+      const double delta = mu - mean;
+      mean += delta * w_mean;
+      m2 += prm.ws_m2[static_cast<int64_t>(rb) * prm.d + c] +
+            delta * delta * (static_cast<double>(n) * w_mean);
+      q += prm.ws_q[static_cast<int64_t>(rb) * prm.d + c];
+      n += nb;
+    }
+    const float gb = static_cast<float>(mean);
+    prm.gbar[c] = gb;
+    a = static_cast<double>(gb) * static_cast<double>(gb);
+    s = m2;
+  }
+  block_reduce3<kWarps>(a, s, q, red);
+  if (threadIdx.x == 0) {
+    double* out = prm.chunk_out + static_cast<int64_t>(blockIdx.x) * 4;
+    out[0] = a;
+    out[1] = s;
+    out[2] = q;
+    out[3] = 0.0;
+  }
+}
+
+// Stand-alone AdamW (Algorithm 1, AdamW lines), in place.
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads)
+    adamw_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,
+                 float* __restrict__ v, int64_t d, const AdamScalars a) {
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
+  if (VEC) {
+    const int64_t nvec = d >> 2;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < nvec;
+         i += stride) {
+      const float4 gg = __ldcs(reinterpret_cast<const float4*>(g) + i);
+      float4 pp = ld_state_16(p + 4 * i), mm = ld_state_16(m + 4 * i), vv = ld_state_16(v + 4 * i);
+      adamw_elem(a, gg.x, pp.x, mm.x, vv.x);
+      adamw_elem(a, gg.y, pp.y, mm.y, vv.y);
+      adamw_elem(a, gg.z, pp.z, mm.z, vv.z);
+      adamw_elem(a, gg.w, pp.w, mm.w, vv.w);
+      st_stream_16(p + 4 * i, pp);
+      st_stream_16(m + 4 * i, mm);
+      st_stream_16(v + 4 * i, vv);
+    }
+    // tail (d % 4 elements) by the first threads of block 0
+    const int64_t t = (nvec << 2) + threadIdx.x;
+    if (blockIdx.x == 0 && t < d) {
+      float pp = p[t], mm = m[t], vv = v[t];
+      adamw_elem(a, g[t], pp, mm, vv);
+      p[t] = pp;
+      m[t] = mm;
+      v[t] = vv;
+    }
+  } else {
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < d;
+         i += stride) {
+      float pp = p[i], mm = m[i], vv = v[i];
+      adamw_elem(a, g[i], pp, mm, vv);
+      p[i] = pp;
+      m[i] = mm;
+      v[i] = vv;
+    }
+  }
+}
+
+}  // namespace absnt
