@@ -1,0 +1,85 @@
+"""Multi-process plumbing (one process per GPU, torch.distributed).
+
+The norm-test + AdamW step is separable per coordinate, so it needs no data-path
+collective: ranks either run independent replicas, or each rank owns an index range of
+the flat vector (the FSDP layout of Sec. 3.3) and only the three fp64 sums per rank
+cross the wire.  This module holds that small host-side logic:
+
+  rank_range          the contiguous index range a rank owns
+  combine_rank_sums   all-gather of {n2, S, Q} per rank, added in rank order on every
+                      rank (so all ranks take the same bit-identical decision), then the
+                      library's host-side decision
+  max_over_ranks      max-reduction used for timing
+"""
+import os
+
+import torch
+import torch.distributed as dist
+
+from . import binding
+
+
+def init_from_env(backend=None):
+    """Initialises the default process group from RANK / WORLD_SIZE / MASTER_* when
+    WORLD_SIZE > 1.  Returns (rank, world_size, local_rank)."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", str(rank)))
+    if world > 1 and not dist.is_initialized():
+        if backend is None:
+            backend = "nccl" if torch.cuda.is_available() else "gloo"
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if backend == "nccl":
+            torch.cuda.set_device(local_rank)
+            dist.init_process_group(backend, device_id=torch.device("cuda", local_rank))
+        else:
+            dist.init_process_group(backend)
+    return rank, world, local_rank
+
+
+def rank_range(d, rank, world):
+    """[lo, hi) of the flat vector owned by `rank`: equal contiguous ranges, the first
+    d % world ranks holding one extra coordinate."""
+    q, r = divmod(int(d), int(world))
+    lo = rank * q + min(rank, r)
+    return lo, lo + q + (1 if rank < r else 0)
+
+
+def combine_rank_sums(n2, S, Q, K, eta, b_cur, device="cpu", group=None):
+    """Each rank passes the sums of its own index range; every rank returns the same
+    dict of totals (added in rank order), statistic, flags and b_next."""
+    local = torch.tensor([n2, S, Q], dtype=torch.float64, device=device)
+    if dist.is_initialized() and dist.get_world_size(group) > 1:
+        parts = [torch.empty_like(local) for _ in range(dist.get_world_size(group))]
+        dist.all_gather(parts, local, group=group)
+    else:
+        parts = [local]
+    tot = [0.0, 0.0, 0.0]
+    for part in parts:  # rank order
+        vals = part.tolist()
+        for j in range(3):
+            tot[j] += vals[j]
+    b_next, T, flags = binding.abs_decide(tot[1], tot[0], K, eta, b_cur)
+    return {"n2": tot[0], "S": tot[1], "Q": tot[2], "T": T, "flags": flags, "b_next": b_next}
+
+
+def barrier(device=None):
+    if dist.is_initialized() and dist.get_world_size() > 1:
+        if device is not None and torch.device(device).type == "cuda":
+            dist.barrier(device_ids=[torch.device(device).index])
+        else:
+            dist.barrier()
+
+
+def max_over_ranks(x, device="cpu"):
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    if dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(x, device="cpu"):
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    if dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())

@@ -1,0 +1,201 @@
+"""CPU-side checks of the C ABI: the library loads, exports every declared symbol, its
+host helpers agree with the hand-worked fixtures, and every invalid-argument path returns
+its status before anything could be launched (no GPU is touched here)."""
+import ctypes
+import json
+import math
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+from paper_2412_21124_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "abs_normtest.h")
+GOLDEN = os.path.join(ROOT, "tests", "golden", "hand_cases.json")
+
+
+@pytest.fixture(scope="module")
+def L():
+    entry.build()
+    return binding.lib()
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(abs_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = declared_functions()
+    assert {"abs_norm_test", "abs_adamw_step", "abs_normtest_adamw",
+            "abs_persample_norm_test"} <= set(names)
+    for n in names:
+        assert hasattr(L, n), "header declares %s but the library does not export it" % n
+
+
+def test_status_strings(L):
+    seen = set()
+    for s in range(0, -7, -1):
+        msg = L.abs_status_string(s).decode()
+        assert msg and msg != "unknown status"
+        seen.add(msg)
+    assert len(seen) == 7
+    assert L.abs_status_string(-99).decode() == "unknown status"
+    assert L.abs_last_cuda_error() == 0
+
+
+def test_decide_matches_hand_cases(L):
+    cases = json.load(open(GOLDEN))["norm_test"]
+    for c in cases:
+        K = len(c["grads"])
+        for dec in c["decisions_worker"]:
+            b_next, T, flags = binding.abs_decide(c["S"], c["n2"], K, c["eta"], dec["b_cur"])
+            assert b_next == dec["b_next"]
+            assert bool(flags & binding.ABS_FLAG_VIOLATED) == dec["violated"]
+        b_next, T, flags = binding.abs_decide(c["S"], c["n2"], K - 1, c["eta"], K)
+        assert b_next == c["b_next_persample"]
+
+
+def test_decide_edge_cases(L):
+    b_next, T, flags = binding.abs_decide(0.0, 0.0, 4, 0.1, 9)
+    assert b_next == 9 and math.isnan(T) and flags == binding.ABS_FLAG_DEGENERATE
+    b_next, T, flags = binding.abs_decide(1.0, 0.0, 4, 0.1, 9)
+    assert b_next == 2 ** 63 - 1 and T == math.inf
+    assert flags == binding.ABS_FLAG_DEGENERATE | binding.ABS_FLAG_VIOLATED
+    for bad in (math.nan, math.inf):
+        b_next, T, flags = binding.abs_decide(bad, 1.0, 4, 0.1, 9)
+        assert b_next == 9 and flags == binding.ABS_FLAG_NONFINITE
+    b_next, T, flags = binding.abs_decide(1.0, 1.0, 2.0, 1e-12, 5)
+    assert b_next == 2 ** 63 - 1 and flags == binding.ABS_FLAG_VIOLATED
+    # ties keep the batch size (the test is satisfied with equality)
+    assert binding.abs_decide(4.0, 8.0, 2.0, 0.25, 4)[0] == 4
+
+
+def test_round_batch_hand_cases(L):
+    for c in json.load(open(GOLDEN))["round_batch"]:
+        for case in c["cases"]:
+            assert binding.abs_round_batch(case["b_next"], case["J"], case["M"]) == case["b"]
+    assert binding.abs_round_batch(0, 4, 4) == -1
+    assert binding.abs_round_batch(5, 0, 4) == -1
+    assert binding.abs_round_batch(5, 4, 0) == -1
+
+
+def test_stats_bytes(L):
+    assert binding.abs_stats_bytes(0, 1) == 0
+    assert binding.abs_stats_bytes(10, 0) == 0
+    assert binding.abs_stats_bytes(10, binding.ABS_MAX_SHARDS + 1) == 0
+    hdr = binding.ABS_STATS_HEADER * 8
+    # one chunk + one spare per shard
+    assert binding.abs_stats_bytes(1, 1) == hdr + 4 * 8 + 2 * 32
+    big = binding.abs_stats_bytes(124_439_808, 8)
+    assert big % 16 == 0 and big < (1 << 20)
+    assert binding.abs_persample_stats_bytes(1, 10) == 0
+    assert binding.abs_persample_stats_bytes(4096, 16384) > 3 * 32 * 16384 * 8
+
+
+# ---- invalid arguments: every path returns its status before any CUDA call ---------------
+FAKE = 0x10000  # a non-null, 16-byte aligned value that is never dereferenced
+
+
+def _nt_args(**over):
+    K = over.pop("K", 2)
+    table = over.pop("table", (ctypes.c_void_p * 32)(*([FAKE] * 32)))
+    a = dict(grads=table, K=K, d=100, dtype=0, offs=None, n_shards=1, eta=0.1, b_cur=8,
+             stats=FAKE, gbar=FAKE, b_next=FAKE, stream=None)
+    a.update(over)
+    return [a[k] for k in ("grads", "K", "d", "dtype", "offs", "n_shards", "eta", "b_cur",
+                           "stats", "gbar", "b_next", "stream")]
+
+
+def _offs(*vals):
+    return (ctypes.c_int64 * len(vals))(*vals)
+
+
+@pytest.mark.parametrize("over,status", [
+    (dict(grads=None), binding.ABS_ERR_NULL),
+    (dict(stats=None), binding.ABS_ERR_NULL),
+    (dict(gbar=None), binding.ABS_ERR_NULL),
+    (dict(b_next=None), binding.ABS_ERR_NULL),
+    (dict(dtype=2), binding.ABS_ERR_DTYPE),
+    (dict(K=0), binding.ABS_ERR_RANGE),
+    (dict(K=33), binding.ABS_ERR_RANGE),
+    (dict(d=0), binding.ABS_ERR_RANGE),
+    (dict(b_cur=0), binding.ABS_ERR_RANGE),
+    (dict(eta=0.0), binding.ABS_ERR_RANGE),
+    (dict(eta=-0.1), binding.ABS_ERR_RANGE),
+    (dict(eta=math.nan), binding.ABS_ERR_RANGE),
+    (dict(eta=math.inf), binding.ABS_ERR_RANGE),
+    (dict(stats=FAKE + 8), binding.ABS_ERR_ALIGN),
+    (dict(gbar=FAKE + 2), binding.ABS_ERR_ALIGN),
+    (dict(b_next=FAKE + 4), binding.ABS_ERR_ALIGN),
+    (dict(table=(ctypes.c_void_p * 32)(FAKE, 0)), binding.ABS_ERR_NULL),
+    (dict(table=(ctypes.c_void_p * 32)(FAKE, FAKE + 2)), binding.ABS_ERR_ALIGN),
+    (dict(offs=_offs(0, 100), n_shards=0), binding.ABS_ERR_RANGE),
+    (dict(offs=_offs(0, 100), n_shards=129), binding.ABS_ERR_RANGE),
+    (dict(offs=_offs(1, 100), n_shards=1), binding.ABS_ERR_SHARDS),
+    (dict(offs=_offs(0, 99), n_shards=1), binding.ABS_ERR_SHARDS),
+    (dict(offs=_offs(0, 60, 50, 100), n_shards=3), binding.ABS_ERR_SHARDS),
+])
+def test_norm_test_rejects(L, over, status):
+    assert L.abs_norm_test(*_nt_args(**over)) == status
+
+
+def _hp(**over):
+    v = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
+    v.update(over)
+    return binding.abs_adamw_hparams(v["lr"], v["beta1"], v["beta2"], v["eps"], v["weight_decay"])
+
+
+@pytest.mark.parametrize("hp,step,status", [
+    (None, 1, binding.ABS_ERR_NULL),
+    (_hp(), 0, binding.ABS_ERR_RANGE),
+    (_hp(beta1=1.0), 1, binding.ABS_ERR_RANGE),
+    (_hp(beta2=-0.1), 1, binding.ABS_ERR_RANGE),
+    (_hp(lr=-1.0), 1, binding.ABS_ERR_RANGE),
+    (_hp(eps=math.nan), 1, binding.ABS_ERR_RANGE),
+    (_hp(weight_decay=math.inf), 1, binding.ABS_ERR_RANGE),
+])
+def test_adamw_and_fused_reject_hparams(L, hp, step, status):
+    ref = ctypes.byref(hp) if hp is not None else None
+    assert L.abs_adamw_step(FAKE, FAKE, FAKE, FAKE, 10, ref, step, None) == status
+    args = _nt_args() [:-1] + [FAKE, FAKE, FAKE, ref, step, None]
+    assert L.abs_normtest_adamw(*args) == status
+
+
+def test_adamw_rejects_pointers(L):
+    hp = _hp()
+    r = ctypes.byref(hp)
+    assert L.abs_adamw_step(None, FAKE, FAKE, FAKE, 10, r, 1, None) == binding.ABS_ERR_NULL
+    assert L.abs_adamw_step(FAKE, FAKE, FAKE, None, 10, r, 1, None) == binding.ABS_ERR_NULL
+    assert L.abs_adamw_step(FAKE, FAKE, FAKE, FAKE, 0, r, 1, None) == binding.ABS_ERR_RANGE
+    assert L.abs_adamw_step(FAKE + 2, FAKE, FAKE, FAKE, 10, r, 1, None) == binding.ABS_ERR_ALIGN
+    # fused: params/m/v required, gbar optional
+    base = _nt_args(gbar=None)[:-1]
+    assert L.abs_normtest_adamw(*(base + [None, FAKE, FAKE, r, 1, None])) == binding.ABS_ERR_NULL
+    assert L.abs_normtest_adamw(*(base + [FAKE, FAKE + 2, FAKE, r, 1, None])) == binding.ABS_ERR_ALIGN
+
+
+@pytest.mark.parametrize("args,status", [
+    ((None, 4, 10, 10, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_NULL),
+    ((FAKE, 4, 10, 10, 0, 0.1, None, FAKE, FAKE, None), binding.ABS_ERR_NULL),
+    ((FAKE, 4, 10, 10, 1, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_DTYPE),
+    ((FAKE, 1, 10, 10, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_RANGE),
+    ((FAKE, 4, 0, 10, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_RANGE),
+    ((FAKE, 4, 10, 9, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_RANGE),
+    ((FAKE, 4, 10, 10, 0, 0.0, FAKE, FAKE, FAKE, None), binding.ABS_ERR_RANGE),
+    ((FAKE + 2, 4, 10, 10, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_ALIGN),
+    ((FAKE, 4, 10, 10, 0, 0.1, FAKE + 8, FAKE, FAKE, None), binding.ABS_ERR_ALIGN),
+])
+def test_persample_rejects(L, args, status):
+    assert L.abs_persample_norm_test(*args) == status
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding._build, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.lib()
