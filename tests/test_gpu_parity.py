@@ -234,7 +234,7 @@ def test_sharding_does_not_change_gbar_or_update():
         outs.append((gbar, p, m, v, absnt.read_stats(stats, n_sh), int(b_next.item())))
     for a, b in zip(outs[0][:4], outs[1][:4]):
         assert torch.equal(a, b)
-    assert outs[0][4]["S"] == pytest.approx(outs[1][4]["S"], rel=1e-12)
+    assert outs[0][4]["S"] == pytest.approx(outs[1][4]["S"], rel=1e-7)  # row grouping differs
     assert outs[0][5] == outs[1][5]
 
 
@@ -271,7 +271,7 @@ def test_identical_buffers_keep_batch_size(K, dtype):
     assert got["S"] == 0.0 and got["T"] == 0.0 and got["flags"] == 0
     assert int(b_next.item()) == 77
     assert torch.equal(gbar, g.float())
-    assert got["Q"] == pytest.approx(K * got["n2"], rel=1e-12)
+    assert got["Q"] == pytest.approx(K * got["n2"], rel=1e-6)  # fp32 row partials
 
 
 def test_degenerate_and_nonfinite_flags():
