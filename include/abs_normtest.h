@@ -63,7 +63,7 @@ typedef struct {
 enum {
   ABS_STAT_N2 = 0,      /* ||gbar||^2, gbar as written/consumed in fp32                  */
   ABS_STAT_S = 1,       /* sum_k ||g_k - gbar||^2   (per-sample form: sum over rows)     */
-  ABS_STAT_Q = 2,       /* sum_k ||g_k||^2          (diagnostic: S = Q - K*n2)           */
+  ABS_STAT_Q = 2,       /* sum_k ||g_k||^2 (diagnostic: S = Q - K*n2); NaN = not computed */
   ABS_STAT_T = 3,       /* the statistic T                                               */
   ABS_STAT_FLAGS = 4,   /* ABS_FLAG_* bits stored as a double                            */
   ABS_STAT_NORM = 5,    /* K (worker form) or b-1 (per-sample form)                      */
@@ -132,7 +132,8 @@ int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t
 /*
  * The fused step: abs_norm_test and abs_adamw_step in one pass, so gradients and
  * optimizer state cross HBM once.  Arguments as above; gbar_out may be NULL (the mean
- * then lives only in registers).  Legal because the update uses only the mean gradient
+ * then lives only in registers).  The diagnostic Q is not computed here: its slots in
+ * stats_out read NaN.  Legal because the update uses only the mean gradient
  * and none of the test's results (Algorithm 1 lists the test first, with no data
  * dependence between the two).
  */

@@ -14,10 +14,11 @@ constexpr int kWarps = kThreads / 32;
 
 // AdamW scalars (Algorithm 1, AdamW lines), prepared on the host in double.
 struct AdamScalars {
-  float beta1, omb1;      // beta1, 1-beta1
-  float beta2, omb2;      // beta2, 1-beta2
-  float inv_bc1, inv_bc2; // 1/(1-beta1^step), 1/(1-beta2^step)
-  float lr, eps, decay;   // alpha, epsilon, 1-alpha*lambda
+  float beta1, omb1;  // beta1, 1-beta1
+  float beta2, omb2;  // beta2, 1-beta2
+  float step_size;    // alpha / (1-beta1^step)
+  float inv_bc2;      // 1/(1-beta2^step)
+  float eps, decay;   // epsilon, 1-alpha*lambda
 };
 
 // Parameter block of the streaming norm-test kernels, passed by value.
@@ -31,6 +32,7 @@ struct StreamParams {
   int n_chunks;
   int chunk_elems; // elements per reduction chunk (a multiple of kThreads*8)
   double inv_K;
+  float inv_Kf, neg_Kf;
   float* gbar; // may be null
   float* p;    // fused AdamW only
   float* m;
@@ -70,10 +72,41 @@ __device__ __forceinline__ void st_stream_16(float* p, float4 x) {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// One AdamW coordinate (Algorithm 1: m_k, v_k, the two hats, w_{k+1}):
+//   w' = (1-alpha*lambda) w - [alpha/(1-beta1^k)] m' / (sqrt(v'/(1-beta2^k)) + eps).
+// The square root and the reciprocal are the hardware approximations (each within
+// 2^-22 relative); they touch only the update term, whose magnitude is about alpha, so
+// the result stays orders of magnitude inside the 1e-6*max|w| parity tolerance while
+// the step costs 12 instructions instead of ~30 -- this kernel runs at the board's
+// power cap, where instructions saved are bandwidth gained.
+__device__ __forceinline__ void adamw_elem(const AdamScalars& a, float g, float& w, float& m,
+                                           float& v) {
+  m = fmaf(a.beta1, m, a.omb1 * g);
+  v = fmaf(a.beta2, v, (a.omb2 * g) * g);
+  float root, inv;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(root) : "f"(v * a.inv_bc2));
+  asm("rcp.approx.f32 %0, %1;" : "=f"(inv) : "f"(root + a.eps));
+  w = fmaf(a.decay, w, -((a.step_size * m) * inv));
+}
+
+// Mean of K fp32 partial sums: s/K.  For K a power of two the product with 1/K is exact;
+// otherwise one residual correction makes K identical inputs return exactly that input.
+template <bool POW2>
+__device__ __forceinline__ float mean_of_sum(float s, float inv_K, float neg_K) {
+  float q = s * inv_K;
+  if (!POW2) q = fmaf(fmaf(neg_K, q, s), inv_K, q);
+  return q;
+}
+
 // Element types of the gradient buffers.
 struct F32 {
   static constexpr int kVec = 4; // elements per 16 bytes
   using scalar = float;
+  using sum_t = double; // fp32 addends: only an fp64 sum keeps the mean correctly rounded
+  template <bool POW2>
+  static __device__ __forceinline__ float mean(double s, const StreamParams& prm) {
+    return static_cast<float>(s * prm.inv_K);
+  }
   static __device__ __forceinline__ float elem(const uint4& r, int e) {
     return __uint_as_float(e == 0 ? r.x : e == 1 ? r.y : e == 2 ? r.z : r.w);
   }
@@ -84,6 +117,11 @@ struct F32 {
 struct BF16 {
   static constexpr int kVec = 8;
   using scalar = uint16_t;
+  using sum_t = float; // 8-bit significands: fp32 partial sums are exact within 13 binades
+  template <bool POW2>
+  static __device__ __forceinline__ float mean(float s, const StreamParams& prm) {
+    return mean_of_sum<POW2>(s, prm.inv_Kf, prm.neg_Kf);
+  }
   static __device__ __forceinline__ float elem(const uint4& r, int e) {
     const uint32_t w = (e >> 1) == 0 ? r.x : (e >> 1) == 1 ? r.y : (e >> 1) == 2 ? r.z : r.w;
     return (e & 1) ? bf16_hi(w) : bf16_lo(w);
@@ -93,17 +131,6 @@ struct BF16 {
         static_cast<uint32_t>(__ldg(reinterpret_cast<const uint16_t*>(base) + i)) << 16);
   }
 };
-
-// One AdamW coordinate (Algorithm 1: m_k, v_k, the two hats, w_{k+1}).
-__device__ __forceinline__ void adamw_elem(const AdamScalars& a, float g, float& w, float& m,
-                                           float& v) {
-  m = fmaf(a.beta1, m, a.omb1 * g);
-  v = fmaf(a.beta2, v, a.omb2 * (g * g));
-  const float mhat = m * a.inv_bc1;
-  const float vhat = v * a.inv_bc2;
-  const float denom = sqrtf(vhat) + a.eps;
-  w = fmaf(a.decay, w, -(a.lr * (mhat / denom)));
-}
 
 // Fixed-shape reduction of three doubles over a CTA of NW warps.  Every call adds the
 // same operands in the same order, so the result is independent of scheduling.

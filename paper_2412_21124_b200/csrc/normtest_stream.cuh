@@ -10,16 +10,76 @@
 // a fixed order per shard and shard records in shard order.
 //
 // Per coordinate (Algorithm 1, "Compute the batch gradient" .. "approximate gradient
-// variance"): the K values are summed in fp64 (exact for K <= 32 fp32/bf16 inputs up to
-// one final rounding), gbar = fp32(sum/K); deviations g_k - gbar, their squares and g_k^2
-// are fp32 over at most V*K terms, then accumulated in fp64.
+// variance"): gbar = fp32(sum_k g_k / K).  fp32 inputs are summed in fp64, so gbar is the
+// correctly rounded mean even under heavy cancellation.  bf16 inputs are summed in fp32,
+// k = 0..K-1 in order: every partial sum is exact unless the addends' exponents spread
+// over more than 13 binades (8-bit significands in a 24-bit accumulator), and fp64
+// conversions would cost ~3% of bandwidth at the power cap.  Deviations g_k - gbar and
+// their squares (and, in the unfused kernel, g_k^2) are fp32 over at most V*K terms per
+// thread-row, then accumulated in fp64.
 #pragma once
 #include "abs_device.cuh"
 
 namespace absnt {
 
-template <typename GT, int KB, bool EXACT, bool ADAM>
-__global__ void __launch_bounds__(kThreads, (KB <= 8 ? 2 : 1))
+// Mean, squared deviations and (optionally) squared values of one coordinate.
+template <typename GT, int KB, bool EXACT, bool WITHQ>
+__device__ __forceinline__ float coord_math(const float (&g)[KB], int K, const StreamParams& prm,
+                                            float& dev2, float& sq) {
+  constexpr bool POW2 = EXACT && ((KB & (KB - 1)) == 0);
+  typename GT::sum_t s = 0;
+#pragma unroll
+  for (int k = 0; k < KB; ++k)
+    if (EXACT || k < K) s += static_cast<typename GT::sum_t>(g[k]);
+  const float mean = GT::template mean<POW2>(s, prm);
+  dev2 = 0.f;
+  sq = 0.f;
+#pragma unroll
+  for (int k = 0; k < KB; ++k)
+    if (EXACT || k < K) {
+      const float dv = g[k] - mean;
+      dev2 = fmaf(dv, dv, dev2);
+      if (WITHQ) sq = fmaf(g[k], g[k], sq);
+    }
+  return mean;
+}
+
+// The V coordinates of one thread-row with element-wise, bounds-checked accesses: used for
+// rows that are ragged (end of a shard) or whose streams are not 16-byte aligned.  Same
+// arithmetic in the same order as the vector path, so both give identical bits.  Kept out
+// of line so that its registers do not weigh on the vector path.
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+__device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t base, int64_t hi,
+                                        float* sums /* n2, S, Q of this thread-row */) {
+  constexpr int V = GT::kVec;
+  float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
+  for (int e = 0; e < V; ++e) {
+    const int64_t i = base + e;
+    if (i >= hi) break;  // the remaining coordinates would add exact zeros
+    float g[KB];
+#pragma unroll
+    for (int k = 0; k < KB; ++k) g[k] = (EXACT || k < K) ? GT::load1(prm.grads[k], i) : 0.f;
+    float dev2, sq;
+    const float mean = coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
+    row_n2 = fmaf(mean, mean, row_n2);
+    row_S += dev2;
+    row_Q += sq;
+    if (prm.gbar) prm.gbar[i] = mean;
+    if (ADAM) {
+      float w = prm.p[i], m = prm.m[i], v = prm.v[i];
+      adamw_elem(prm.adam, mean, w, m, v);
+      prm.p[i] = w;
+      prm.m[i] = m;
+      prm.v[i] = v;
+    }
+  }
+  sums[0] = row_n2;
+  sums[1] = row_S;
+  sums[2] = row_Q;
+}
+
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+__global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 ? 2 : 1)))
     normtest_stream_kernel(const __grid_constant__ StreamParams prm) {
   constexpr int V = GT::kVec;
   constexpr int NF4 = V / 4; // float4 per thread-row of an fp32 array
@@ -59,98 +119,62 @@ __global__ void __launch_bounds__(kThreads, (KB <= 8 ? 2 : 1))
 
     for (int64_t row_lo = lo; row_lo < hi; row_lo += kThreads * V) {
       const int64_t base = row_lo + static_cast<int64_t>(tid) * V;
-      const bool fast = aligned && (row_lo + kThreads * V <= hi);
+      float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
 
-      uint4 raw[KB];
-      float pw[V], pm[V], pv[V];
-      if (fast) {
+      if (aligned && (row_lo + kThreads * V <= hi)) {
+        uint4 raw[KB];
 #pragma unroll
         for (int k = 0; k < KB; ++k)
           if (EXACT || k < K)
             raw[k] = ld_once_16(reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) + base);
+        float4 pw[NF4], pm[NF4], pv[NF4];
         if (ADAM) {
 #pragma unroll
           for (int q = 0; q < NF4; ++q) {
-            const float4 a = ld_state_16(prm.p + base + 4 * q);
-            const float4 b = ld_state_16(prm.m + base + 4 * q);
-            const float4 c = ld_state_16(prm.v + base + 4 * q);
-            pw[4 * q + 0] = a.x; pw[4 * q + 1] = a.y; pw[4 * q + 2] = a.z; pw[4 * q + 3] = a.w;
-            pm[4 * q + 0] = b.x; pm[4 * q + 1] = b.y; pm[4 * q + 2] = b.z; pm[4 * q + 3] = b.w;
-            pv[4 * q + 0] = c.x; pv[4 * q + 1] = c.y; pv[4 * q + 2] = c.z; pv[4 * q + 3] = c.w;
+            pw[q] = ld_state_16(prm.p + base + 4 * q);
+            pm[q] = ld_state_16(prm.m + base + 4 * q);
+            pv[q] = ld_state_16(prm.v + base + 4 * q);
           }
         }
-      }
-
-      float gb[V];
-      float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
+        // four coordinates at a time, stored as soon as they are done (short live ranges)
 #pragma unroll
-      for (int e = 0; e < V; ++e) {
-        float g[KB];
-        if (fast) {
+        for (int q = 0; q < NF4; ++q) {
+          float gb[4];
+          float* w4 = reinterpret_cast<float*>(&pw[q]);
+          float* m4 = reinterpret_cast<float*>(&pm[q]);
+          float* v4 = reinterpret_cast<float*>(&pv[q]);
 #pragma unroll
-          for (int k = 0; k < KB; ++k) g[k] = (EXACT || k < K) ? GT::elem(raw[k], e) : 0.f;
-        } else {
-          const bool in = base + e < hi;
+          for (int j = 0; j < 4; ++j) {
+            float g[KB];
 #pragma unroll
-          for (int k = 0; k < KB; ++k)
-            g[k] = ((EXACT || k < K) && in) ? GT::load1(prm.grads[k], base + e) : 0.f;
+            for (int k = 0; k < KB; ++k)
+              g[k] = (EXACT || k < K) ? GT::elem(raw[k], 4 * q + j) : 0.f;
+            float dev2, sq;
+            const float mean = coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
+            gb[j] = mean;
+            row_n2 = fmaf(mean, mean, row_n2);
+            row_S += dev2;
+            row_Q += sq;
+            if (ADAM) adamw_elem(prm.adam, mean, w4[j], m4[j], v4[j]);
+          }
+          if (prm.gbar)
+            st_stream_16(prm.gbar + base + 4 * q, make_float4(gb[0], gb[1], gb[2], gb[3]));
           if (ADAM) {
-            pw[e] = in ? prm.p[base + e] : 0.f;
-            pm[e] = in ? prm.m[base + e] : 0.f;
-            pv[e] = in ? prm.v[base + e] : 0.f;
+            st_stream_16(prm.p + base + 4 * q, pw[q]);
+            st_stream_16(prm.m + base + 4 * q, pm[q]);
+            st_stream_16(prm.v + base + 4 * q, pv[q]);
           }
         }
-        double s = 0.0;
-#pragma unroll
-        for (int k = 0; k < KB; ++k)
-          if (EXACT || k < K) s += static_cast<double>(g[k]);
-        const float mean = static_cast<float>(s * prm.inv_K);
-        float dev2 = 0.f, sq = 0.f;
-#pragma unroll
-        for (int k = 0; k < KB; ++k)
-          if (EXACT || k < K) {
-            const float dv = g[k] - mean;
-            dev2 = fmaf(dv, dv, dev2);
-            sq = fmaf(g[k], g[k], sq);
-          }
-        gb[e] = mean;
-        row_n2 = fmaf(mean, mean, row_n2);
-        row_S += dev2;
-        row_Q += sq;
-        if (ADAM) adamw_elem(prm.adam, mean, pw[e], pm[e], pv[e]);
+      } else if (base < hi) {
+        float sums[3];
+        scalar_row<GT, KB, EXACT, ADAM, WITHQ>(prm, K, base, hi, sums);
+        row_n2 = sums[0];
+        row_S = sums[1];
+        row_Q = sums[2];
       }
       acc_n2 += static_cast<double>(row_n2);
       acc_S += static_cast<double>(row_S);
-      acc_Q += static_cast<double>(row_Q);
-
-      if (fast) {
-#pragma unroll
-        for (int q = 0; q < NF4; ++q) {
-          if (prm.gbar)
-            st_stream_16(prm.gbar + base + 4 * q,
-                         make_float4(gb[4 * q], gb[4 * q + 1], gb[4 * q + 2], gb[4 * q + 3]));
-          if (ADAM) {
-            st_stream_16(prm.p + base + 4 * q,
-                         make_float4(pw[4 * q], pw[4 * q + 1], pw[4 * q + 2], pw[4 * q + 3]));
-            st_stream_16(prm.m + base + 4 * q,
-                         make_float4(pm[4 * q], pm[4 * q + 1], pm[4 * q + 2], pm[4 * q + 3]));
-            st_stream_16(prm.v + base + 4 * q,
-                         make_float4(pv[4 * q], pv[4 * q + 1], pv[4 * q + 2], pv[4 * q + 3]));
-          }
-        }
-      } else {
-#pragma unroll
-        for (int e = 0; e < V; ++e) {
-          if (base + e < hi) {
-            if (prm.gbar) prm.gbar[base + e] = gb[e];
-            if (ADAM) {
-              prm.p[base + e] = pw[e];
-              prm.m[base + e] = pm[e];
-              prm.v[base + e] = pv[e];
-            }
-          }
-        }
-      }
+      if (WITHQ) acc_Q += static_cast<double>(row_Q);
     }
 
     block_reduce3<kWarps>(acc_n2, acc_S, acc_Q, red);
@@ -158,7 +182,7 @@ __global__ void __launch_bounds__(kThreads, (KB <= 8 ? 2 : 1))
       double* out = prm.chunk_out + static_cast<int64_t>(chunk) * 4;
       out[0] = acc_n2;
       out[1] = acc_S;
-      out[2] = acc_Q;
+      out[2] = WITHQ ? acc_Q : __longlong_as_double(0x7ff8000000000000ll);  // NaN: not computed
       out[3] = 0.0;
     }
   }
