@@ -43,7 +43,8 @@ typedef enum {
   ABS_ERR_SHARDS = -3, /* shard_offsets not non-decreasing, or ends are not 0 and d    */
   ABS_ERR_ALIGN = -4,  /* a buffer is not aligned to its element size                  */
   ABS_ERR_DTYPE = -5,  /* dtype is not an abs_dtype                                    */
-  ABS_ERR_CUDA = -6    /* a CUDA call failed; see abs_last_cuda_error()                */
+  ABS_ERR_CUDA = -6,   /* a CUDA call failed; see abs_last_cuda_error()                */
+  ABS_ERR_TOO_LARGE = -7 /* the problem needs more built-in scratch than the library holds */
 } abs_status;
 
 enum { ABS_MAX_WORKERS = 32, ABS_MAX_SHARDS = 128 };
@@ -142,6 +143,48 @@ int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dty
                        void* stats_out, float* gbar_out, int64_t* b_next_out, float* params,
                        float* m, float* v, const abs_adamw_hparams* hparams, int64_t step,
                        abs_stream_t stream);
+
+/*
+ * abs_normtest_adamw for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a deployment convenience, not part of the method.)
+ *
+ * Who needs it.  abs_normtest_adamw keeps its per-chunk partial sums in the tail of
+ * stats_out, whose size grows with d, so the caller has to size and allocate that buffer
+ * for every new problem size.  Some callers cannot: code that runs inside a region where
+ * cudaMalloc is forbidden or would stall everything (a plugin's execute hook, a callback
+ * on a latency-critical serving path, a process whose device memory is entirely owned by
+ * another allocator), or a host that only has a fixed, small status buffer to offer.
+ * This variant needs nothing that grows with d: the partial sums go to an array that is
+ * part of the library image (ABS_NOALLOC_MAX_CHUNKS records of 32 bytes = 4 MiB, resident
+ * on every GPU that loads the library until the process exits).  The call itself performs
+ * no cudaMalloc/cudaFree and calls no allocating routine.
+ *
+ * Arguments, results and status codes are those of abs_normtest_adamw, except:
+ *   stats_out   device, only (ABS_STATS_HEADER + n_shards*ABS_SHARD_STRIDE) doubles
+ *               (header and shard records; no scratch tail), 16-byte aligned
+ *   limit       ceil(d/c) + n_shards must not exceed ABS_NOALLOC_MAX_CHUNKS, where c = 16384
+ *               for d >= 2^23 and 4096 below (any d up to about 2.1e9); larger problems
+ *               return ABS_ERR_TOO_LARGE and launch nothing
+ * Results are bit-identical to abs_normtest_adamw on the same inputs.
+ *
+ * Shared state.  All calls on one device use the same built-in array.  Nothing in it has
+ * to be cleared between calls: every record the final reduction reads is written earlier
+ * in the same call, so stale contents of a previous call are never observed.  But two
+ * calls whose GPU work overlaps on one device (different streams, or several host threads)
+ * race on it and produce undefined statistics: keep them on one stream or otherwise
+ * ordered.
+ * First call.  The first call on each device looks up the device address of the built-in
+ * array (cudaGetSymbolAddress, with that device current; this may also trigger the lazy
+ * load of the library's device code).  Make that first call outside of any stream
+ * capture; later calls on the same device only launch kernels.
+ */
+enum { ABS_NOALLOC_MAX_CHUNKS = 131072 };
+int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                               const int64_t* shard_offsets, int n_shards, double eta,
+                               int64_t b_cur, void* stats_out, float* gbar_out,
+                               int64_t* b_next_out, float* params, float* m, float* v,
+                               const abs_adamw_hparams* hparams, int64_t step,
+                               abs_stream_t stream);
 
 /*
  * Approximate norm test on per-sample gradients (Eq. 3, the Var definition before it,

@@ -16,6 +16,8 @@ ABS_F32, ABS_BF16 = 0, 1
 ABS_OK = 0
 ABS_ERR_NULL, ABS_ERR_RANGE, ABS_ERR_SHARDS, ABS_ERR_ALIGN, ABS_ERR_DTYPE, ABS_ERR_CUDA = (
     -1, -2, -3, -4, -5, -6)
+ABS_ERR_TOO_LARGE = -7
+ABS_NOALLOC_MAX_CHUNKS = 131072
 ABS_MAX_WORKERS, ABS_MAX_SHARDS = 32, 128
 (ABS_STAT_N2, ABS_STAT_S, ABS_STAT_Q, ABS_STAT_T, ABS_STAT_FLAGS, ABS_STAT_NORM,
  ABS_STAT_NCHUNKS) = range(7)
@@ -64,6 +66,8 @@ def lib():
     L.abs_normtest_adamw.restype = cint
     L.abs_normtest_adamw.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64, ptr, ptr, ptr,
                                      ptr, ptr, ptr, ptr, i64, ptr]
+    L.abs_normtest_adamw_noalloc.restype = cint
+    L.abs_normtest_adamw_noalloc.argtypes = list(L.abs_normtest_adamw.argtypes)
     L.abs_persample_norm_test.restype = cint
     L.abs_persample_norm_test.argtypes = [ptr, i64, i64, i64, cint, dbl, ptr, ptr, ptr, ptr]
     L.abs_decide.restype = i64
@@ -193,6 +197,32 @@ def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, param
                                   v.data_ptr(), ctypes.byref(hp), int(step), _stream(stream))
     if rc != ABS_OK:
         raise AbsError(rc, "abs_normtest_adamw")
+
+
+def abs_normtest_adamw_noalloc(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v,
+                               hparams, step, shard_offsets=None, stream=None):
+    """abs_normtest_adamw for callers that cannot allocate device memory: `stats_out` only
+    needs ABS_STATS_HEADER + n_shards*ABS_SHARD_STRIDE doubles, the per-chunk records live
+    in an array built into the library (shared by all calls on a device, so calls whose GPU
+    work overlaps race).  Raises AbsError(ABS_ERR_TOO_LARGE) beyond ABS_NOALLOC_MAX_CHUNKS
+    chunks.  Make the first call on a device outside of stream capture."""
+    table, K, d, code = _grad_table(grads)
+    offs, n_shards = _offsets(shard_offsets)
+    for t, name in ((params, "params"), (m, "m"), (v, "v")):
+        _check_f32_vec(t, d, name)
+    if gbar_out is not None:
+        _check_f32_vec(gbar_out, d, "gbar_out")
+    if stats_out.numel() * stats_out.element_size() < 8 * (ABS_STATS_HEADER + n_shards * ABS_SHARD_STRIDE):
+        raise ValueError("stats_out is smaller than header + shard records")
+    hp = _hparams(hparams)
+    rc = lib().abs_normtest_adamw_noalloc(table, K, d, code, offs, n_shards, float(eta),
+                                          int(b_cur), stats_out.data_ptr(),
+                                          gbar_out.data_ptr() if gbar_out is not None else None,
+                                          b_next_out.data_ptr(), params.data_ptr(), m.data_ptr(),
+                                          v.data_ptr(), ctypes.byref(hp), int(step),
+                                          _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_normtest_adamw_noalloc")
 
 
 def abs_persample_norm_test(G, eta, stats_out, gbar_out, b_next_out, stream=None):

@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 
 #include "abs_device.cuh"
 #include "normtest_stream.cuh"
@@ -358,6 +359,9 @@ const char* abs_status_string(int status) {
     case ABS_ERR_ALIGN: return "a buffer is not aligned to its element size";
     case ABS_ERR_DTYPE: return "unsupported dtype";
     case ABS_ERR_CUDA: return "a CUDA call failed (see abs_last_cuda_error)";
+    case ABS_ERR_TOO_LARGE:
+      return "the problem needs more chunk records than the built-in scratch holds "
+             "(ABS_NOALLOC_MAX_CHUNKS); use abs_normtest_adamw with a caller-sized stats_out";
     default: return "unknown status";
   }
 }
@@ -365,3 +369,111 @@ const char* abs_status_string(int status) {
 int abs_last_cuda_error(void) { return g_last_cuda_error; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------
+// abs_normtest_adamw_noalloc: the fused step with its chunk records in an array that is
+// part of the library image, for callers that cannot allocate device memory.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+// One {n2, S, Q, 0} record per chunk.  Lives in every device's copy of the module.
+static __device__ __align__(256) double g_noalloc_chunk_records[ABS_NOALLOC_MAX_CHUNKS * 4];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+double* g_noalloc_device_ptr[kMaxDevices] = {};  // device address of the array, per device
+
+// In host code `g_noalloc_chunk_records` is only a handle for the runtime, not an address
+// a kernel could use: the device address is looked up once per device (with that device
+// current) and cached.
+int noalloc_records_for_current_device(double** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= kMaxDevices) return ABS_ERR_RANGE;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_device_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_chunk_records);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_noalloc_device_ptr[dev] = static_cast<double*>(p);
+  }
+  *out = g_noalloc_device_ptr[dev];
+  return ABS_OK;
+}
+
+}  // namespace
+
+extern "C" int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64_t d,
+                                          abs_dtype dtype, const int64_t* shard_offsets,
+                                          int n_shards, double eta, int64_t b_cur,
+                                          void* stats_out, float* gbar_out, int64_t* b_next_out,
+                                          float* params, float* m, float* v,
+                                          const abs_adamw_hparams* hparams, int64_t step,
+                                          abs_stream_t stream) {
+  if (!grads || !stats_out || !b_next_out || !params || !m || !v) return ABS_ERR_NULL;
+  if (dtype != ABS_F32 && dtype != ABS_BF16) return ABS_ERR_DTYPE;
+  if (K < 1 || K > ABS_MAX_WORKERS || d < 1 || b_cur < 1) return ABS_ERR_RANGE;
+  if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
+  int rc = check_hparams(hparams, step);
+  if (rc != ABS_OK) return rc;
+  const size_t esz = (dtype == ABS_F32) ? 4 : 2;
+  for (int k = 0; k < K; ++k) {
+    if (!grads[k]) return ABS_ERR_NULL;
+    if (misaligned(grads[k], esz)) return ABS_ERR_ALIGN;
+  }
+  if (misaligned(stats_out, 16) || misaligned(b_next_out, 8)) return ABS_ERR_ALIGN;
+  if (gbar_out && misaligned(gbar_out, 4)) return ABS_ERR_ALIGN;
+  if (misaligned(params, 4) || misaligned(m, 4) || misaligned(v, 4)) return ABS_ERR_ALIGN;
+
+  Layout L;
+  rc = make_layout(d, shard_offsets, n_shards, &L);
+  if (rc != ABS_OK) return rc;
+  if (L.n_chunks > ABS_NOALLOC_MAX_CHUNKS) return ABS_ERR_TOO_LARGE;
+
+  double* records = nullptr;
+  rc = noalloc_records_for_current_device(&records);
+  if (rc != ABS_OK) return rc;
+
+  StreamParams prm;
+  std::memset(&prm, 0, sizeof prm);
+  for (int k = 0; k < K; ++k) prm.grads[k] = grads[k];
+  std::memcpy(prm.shard_off, L.shard_off, sizeof(int64_t) * (L.n_shards + 1));
+  std::memcpy(prm.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
+  prm.d = d;
+  prm.K = K;
+  prm.n_shards = L.n_shards;
+  prm.n_chunks = L.n_chunks;
+  prm.chunk_elems = L.chunk_elems;
+  prm.inv_K = 1.0 / static_cast<double>(K);
+  prm.inv_Kf = static_cast<float>(prm.inv_K);
+  prm.neg_Kf = -static_cast<float>(K);
+  prm.gbar = gbar_out;
+  prm.p = params;
+  prm.m = m;
+  prm.v = v;
+  prm.chunk_out = records;  // every record read below is written by this launch first
+  prm.adam = make_adam(hparams, step);
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = (dtype == ABS_F32) ? launch_stream<F32, true>(prm, st)
+                                     : launch_stream<BF16, true>(prm, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+
+  FinalizeParams fp;
+  std::memset(&fp, 0, sizeof fp);
+  fp.chunk_in = records;
+  std::memcpy(fp.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
+  fp.n_shards = L.n_shards;
+  fp.n_chunks = L.n_chunks;
+  fp.stats = static_cast<double*>(stats_out);
+  fp.b_next = b_next_out;
+  fp.eta = eta;
+  fp.norm = static_cast<double>(K);
+  fp.b_cur = b_cur;
+  finalize_kernel<<<1, kFinalizeThreads, 0, st>>>(fp);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return ABS_OK;
+}
+
