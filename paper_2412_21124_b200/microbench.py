@@ -1,0 +1,145 @@
+"""Per-call micro-benchmark of the library on synthetic inputs (one JSON line per point).
+
+  python -m paper_2412_21124_b200.microbench --call fused --d 33554432 --K 8 --dtype bf16
+  python -m paper_2412_21124_b200.microbench --sweep            # the d x K x dtype grid
+
+Timing: CUDA events on the launching stream around `steps` back-to-back calls after
+`warmup` calls.  Points whose working set is smaller than twice the L2 rotate over several
+independent buffer sets so that every call reads cold data.  GB/s counts algorithmic bytes:
+fused (K*s + 24) per coordinate (+4 with --gbar), normtest K*s + 4, adamw 28, persample 4
+per matrix element.
+"""
+import argparse
+import json
+import sys
+
+import torch
+
+from . import binding as B
+from . import synth
+
+HP = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
+L2_BYTES = 126 * 1024 * 1024
+SWEEP_D = (1_048_576, 16_777_216, 124_439_808, 400_000_000, 1_235_814_400)
+SWEEP_K = (2, 4, 8, 16, 32)
+MEM_CAP = 160e9
+
+
+def _sizes(d):
+    if d == 124_439_808:
+        return synth.gpt2_small_tensor_sizes()
+    return synth.pseudo_tensor_sizes(d)
+
+
+def bytes_per_call(call, d, K, esz, gbar, b):
+    if call == "fused":
+        return (K * esz + 24 + (4 if gbar else 0)) * d
+    if call == "normtest":
+        return (K * esz + 4) * d
+    if call == "adamw":
+        return 28 * d
+    return 4 * b * d
+
+
+def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b=4096, dev="cuda"):
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    esz = 2 if dtype == "bf16" else 4
+    nbytes = bytes_per_call(call, d, K, esz, gbar, b)
+    n_sets = 1 if nbytes >= 2 * L2_BYTES else -(-2 * L2_BYTES // nbytes) + 1
+    offs = synth.equal_shard_offsets(d, n_shards) if n_shards > 1 else None
+    sets = []
+    for i in range(n_sets):
+        s = {}
+        if call in ("fused", "normtest"):
+            sizes = _sizes(d)
+            sig = synth.per_tensor_sigma(sizes, 11)
+            s["grads"] = synth.worker_grads(sizes, K, tdt, 100 + i, dev, sigma=sig)
+            s["stats"] = B.alloc_stats(d, n_shards, dev)
+        if call in ("fused", "adamw"):
+            s["p"], s["m"], s["v"] = synth.adam_state(d, 200 + i, dev, zero_moments=False)
+        if call in ("normtest", "adamw") or gbar:
+            s["gbar"] = torch.zeros(d, dtype=torch.float32, device=dev)
+            if call == "adamw":
+                s["gbar"].normal_().mul_(0.02)
+        if call == "persample":
+            s["G"] = torch.empty(b, d, dtype=torch.float32, device=dev).normal_().mul_(0.3)
+            s["stats"] = B.alloc_persample_stats(b, d, dev)
+            s["gbar"] = torch.zeros(d, dtype=torch.float32, device=dev)
+        s["b_next"] = torch.zeros(1, dtype=torch.int64, device=dev)
+        sets.append(s)
+
+    def one(i):
+        s = sets[i % n_sets]
+        if call == "fused":
+            B.abs_normtest_adamw(s["grads"], 0.1, 512, s["stats"], s.get("gbar"), s["b_next"],
+                                 s["p"], s["m"], s["v"], HP, 100 + i, shard_offsets=offs)
+        elif call == "normtest":
+            B.abs_norm_test(s["grads"], 0.1, 512, s["stats"], s["gbar"], s["b_next"],
+                            shard_offsets=offs)
+        elif call == "adamw":
+            B.abs_adamw_step(s["p"], s["gbar"], s["m"], s["v"], HP, 100 + i)
+        else:
+            B.abs_persample_norm_test(s["G"], 0.1, s["stats"], s["gbar"], s["b_next"])
+
+    for i in range(warmup):
+        one(i)
+    torch.cuda.synchronize()
+    if steps is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        one(0)
+        e1.record()
+        torch.cuda.synchronize()
+        est = max(e0.elapsed_time(e1), 1e-3)
+        steps = int(max(10, min(400, 300.0 / est)))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stream = torch.cuda.current_stream()
+    e0.record(stream)
+    for i in range(steps):
+        one(warmup + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    out = {"call": call, "d": d, "K": K, "dtype": dtype, "n_shards": n_shards, "gbar": bool(gbar),
+           "steps": steps, "buffer_sets": n_sets, "ms": ms, "bytes": nbytes,
+           "GBps": nbytes / (ms * 1e-3) / 1e9}
+    if call == "persample":
+        out["b"] = b
+    return out
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--call", choices=["fused", "normtest", "adamw", "persample"], default="fused")
+    ap.add_argument("--d", type=int, default=33_554_432)
+    ap.add_argument("--K", type=int, default=8)
+    ap.add_argument("--dtype", choices=["bf16", "f32"], default="bf16")
+    ap.add_argument("--shards", type=int, default=1)
+    ap.add_argument("--b", type=int, default=4096, help="rows of the per-sample matrix")
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--gbar", action="store_true", help="fused: also write gbar")
+    ap.add_argument("--sweep", action="store_true", help="fused call over the d x K x dtype grid")
+    args = ap.parse_args(argv)
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device (there is no CPU fallback)")
+    B.lib()
+    if not args.sweep:
+        print(json.dumps(run_point(args.call, args.d, args.K, args.dtype, args.shards, args.steps,
+                                   args.warmup, args.gbar, args.b)), flush=True)
+        return
+    for dtype in ("bf16", "f32"):
+        esz = 2 if dtype == "bf16" else 4
+        for d in SWEEP_D:
+            for K in SWEEP_K:
+                if K * d * esz + 16 * d > MEM_CAP:
+                    print(json.dumps({"call": "fused", "d": d, "K": K, "dtype": dtype,
+                                      "skipped": "K*d*s + 16*d exceeds 160 GB"}), flush=True)
+                    continue
+                r = run_point("fused", d, K, dtype, steps=args.steps, warmup=args.warmup)
+                print(json.dumps(r), flush=True)
+                torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main(sys.argv[1:])
