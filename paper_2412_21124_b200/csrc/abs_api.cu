@@ -5,6 +5,7 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <utility>
 
 #include "abs_device.cuh"
 #include "normtest_stream.cuh"
@@ -53,6 +54,23 @@ AdamScalars make_adam(const abs_adamw_hparams* h, int64_t step) {
   return a;
 }
 
+// Launch with the programmatic-stream-serialization attribute (see grid_dependency_wait).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st,
+                       Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 bool misaligned(const void* p, size_t a) {
   return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
 }
@@ -98,22 +116,21 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
   const int grid = prm.n_chunks;
   const int K = prm.K;
 #define ABS_LAUNCH(KB, EXACT) \
-  normtest_stream_kernel<GT, KB, EXACT, ADAM, !ADAM><<<grid, kThreads, 0, st>>>(prm)
+  launch_pdl(normtest_stream_kernel<GT, KB, EXACT, ADAM, !ADAM>, dim3(grid), dim3(kThreads), st, prm)
   switch (K) {
-    case 1: ABS_LAUNCH(1, true); break;
-    case 2: ABS_LAUNCH(2, true); break;
-    case 3: ABS_LAUNCH(3, true); break;
-    case 4: ABS_LAUNCH(4, true); break;
-    case 8: ABS_LAUNCH(8, true); break;
-    case 16: ABS_LAUNCH(16, true); break;
-    case 32: ABS_LAUNCH(32, true); break;
+    case 1: return ABS_LAUNCH(1, true);
+    case 2: return ABS_LAUNCH(2, true);
+    case 3: return ABS_LAUNCH(3, true);
+    case 4: return ABS_LAUNCH(4, true);
+    case 8: return ABS_LAUNCH(8, true);
+    case 16: return ABS_LAUNCH(16, true);
+    case 32: return ABS_LAUNCH(32, true);
     default:
-      if (K < 8) ABS_LAUNCH(8, false);
-      else if (K < 16) ABS_LAUNCH(16, false);
-      else ABS_LAUNCH(32, false);
+      if (K < 8) return ABS_LAUNCH(8, false);
+      if (K < 16) return ABS_LAUNCH(16, false);
+      return ABS_LAUNCH(32, false);
   }
 #undef ABS_LAUNCH
-  return cudaGetLastError();
 }
 
 int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
@@ -188,8 +205,7 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   fp.eta = eta;
   fp.norm = static_cast<double>(K);
   fp.b_cur = b_cur;
-  finalize_kernel<<<1, kFinalizeThreads, 0, st>>>(fp);
-  e = cudaGetLastError();
+  e = launch_pdl(finalize_kernel, dim3(1), dim3(kFinalizeThreads), st, fp);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -245,16 +261,16 @@ int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t
   const AdamScalars a = make_adam(hparams, step);
   const bool vec = !(misaligned(params, 16) || misaligned(gbar, 16) || misaligned(m, 16) ||
                      misaligned(v, 16));
+  // one CTA per 2048 vectors (two per thread), so CTAs retire and are replaced
+  // continuously, as in the streaming kernels; a grid-stride loop covers huge d
   const int64_t work = vec ? (d + 3) / 4 : d;
-  int64_t blocks = (work + kThreads - 1) / kThreads;
-  const int64_t cap = 148 * 16;
+  int64_t blocks = (work + 2 * kThreads - 1) / (2 * kThreads);
+  const int64_t cap = int64_t{1} << 22;
   if (blocks > cap) blocks = cap;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (vec)
-    adamw_kernel<true><<<static_cast<int>(blocks), kThreads, 0, st>>>(params, gbar, m, v, d, a);
-  else
-    adamw_kernel<false><<<static_cast<int>(blocks), kThreads, 0, st>>>(params, gbar, m, v, d, a);
-  const cudaError_t e = cudaGetLastError();
+  const dim3 grid(static_cast<unsigned>(blocks)), block(kThreads);
+  const cudaError_t e = vec ? launch_pdl(adamw_kernel<true>, grid, block, st, params, gbar, m, v, d, a)
+                            : launch_pdl(adamw_kernel<false>, grid, block, st, params, gbar, m, v, d, a);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -291,19 +307,19 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool vec = !misaligned(G, 16) && (ld % 4 == 0);
+  cudaError_t e;
   if (vec) {
     const int64_t cols = (d + 3) / 4;
     dim3 grid(static_cast<unsigned>((cols + kThreads - 1) / kThreads),
               static_cast<unsigned>(nrb));
-    persample_partial_kernel<4><<<grid, kThreads, 0, st>>>(prm);
+    e = launch_pdl(persample_partial_kernel<4>, grid, dim3(kThreads), st, prm);
   } else {
     dim3 grid(static_cast<unsigned>(n_chunks64), static_cast<unsigned>(nrb));
-    persample_partial_kernel<1><<<grid, kThreads, 0, st>>>(prm);
+    e = launch_pdl(persample_partial_kernel<1>, grid, dim3(kThreads), st, prm);
   }
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
-  persample_merge_kernel<<<static_cast<int>(n_chunks64), kThreads, 0, st>>>(prm);
-  e = cudaGetLastError();
+  e = launch_pdl(persample_merge_kernel, dim3(static_cast<unsigned>(n_chunks64)), dim3(kThreads),
+                 st, prm);
   if (e != cudaSuccess) return cuda_fail(e);
 
   FinalizeParams fp;
@@ -318,8 +334,7 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
   fp.eta = eta;
   fp.norm = static_cast<double>(b - 1);
   fp.b_cur = b;
-  finalize_kernel<<<1, kFinalizeThreads, 0, st>>>(fp);
-  e = cudaGetLastError();
+  e = launch_pdl(finalize_kernel, dim3(1), dim3(kFinalizeThreads), st, fp);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -471,8 +486,7 @@ extern "C" int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64
   fp.eta = eta;
   fp.norm = static_cast<double>(K);
   fp.b_cur = b_cur;
-  finalize_kernel<<<1, kFinalizeThreads, 0, st>>>(fp);
-  e = cudaGetLastError();
+  e = launch_pdl(finalize_kernel, dim3(1), dim3(kFinalizeThreads), st, fp);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }

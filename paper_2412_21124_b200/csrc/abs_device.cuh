@@ -52,6 +52,17 @@ struct FinalizeParams {
   int64_t b_cur;
 };
 
+// ---- programmatic dependent launch ---------------------------------------------------
+// Every kernel of the library is launched with the programmatic-stream-serialization
+// attribute and executes this wait before its first global-memory access.  The launch
+// latency and the index arithmetic of a kernel then overlap the tail of its predecessor
+// in the stream, while the wait itself returns only once that predecessor has completed
+// and its writes are visible -- so ordering is exactly that of an ordinary launch.
+// Without the attribute the instruction is a no-op.
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- streaming memory access --------------------------------------------------------
 // Gradients are read exactly once and never written: non-coherent path, no L1 allocation.
 __device__ __forceinline__ uint4 ld_once_16(const void* p) {

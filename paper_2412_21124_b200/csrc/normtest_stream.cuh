@@ -87,6 +87,7 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 
 
   const int K = EXACT ? KB : prm.K;
   const int tid = threadIdx.x;
+  bool waited = false;
 
   for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
     // shard that owns this chunk: largest s with chunk_prefix[s] <= chunk
@@ -114,6 +115,10 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 
       bits |= reinterpret_cast<uintptr_t>(prm.v) + static_cast<uintptr_t>(lo) * 4;
     }
     const bool aligned = (bits & 15) == 0;
+    if (!waited) {  // everything above used kernel parameters only
+      grid_dependency_wait();
+      waited = true;
+    }
 
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
 
@@ -188,39 +193,97 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 
   }
 }
 
-// One CTA.  Per shard: thread t adds chunk triples t, t+1024, ... of that shard in order,
-// then a fixed tree over the CTA; thread 0 adds shard records in shard order, takes the
-// decision (Algorithm 1: statistic T_k and the If/Else) and writes header + records.
-constexpr int kFinalizeThreads = 1024;
+// One CTA of kFinalizeThreads threads.  Shards with many chunks are reduced by the whole
+// CTA (thread t adds records t, t+T, ... in that order, four loads in flight, then a fixed
+// tree); shards with few chunks by one warp each.  Thread 0 then adds the shard records
+// in shard order, takes the decision (Algorithm 1: statistic T_k and the If/Else) and
+// writes the header.  The shape of every sum depends only on the chunk counts.
+constexpr int kFinalizeThreads = 256;
+constexpr int kFinalizeWarps = kFinalizeThreads / 32;
+constexpr int kSmallShardChunks = 512;
+
+__device__ __forceinline__ void add_record(const double* chunk_in, int ch, double& a, double& b,
+                                           double& c) {
+  const double2* rec = reinterpret_cast<const double2*>(chunk_in + static_cast<int64_t>(ch) * 4);
+  const double2 t0 = rec[0], t1 = rec[1];
+  a += t0.x;
+  b += t0.y;
+  c += t1.x;
+}
+
+// records c0 + first, c0 + first + stride, ... (< c1), in order, four loads in flight
+__device__ __forceinline__ void strided_records(const double* chunk_in, int c0, int c1, int first,
+                                                int stride, double& a, double& b, double& c) {
+  int ch = c0 + first;
+  for (; ch + 3 * stride < c1; ch += 4 * stride) {
+    double2 t[8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const double2* rec =
+          reinterpret_cast<const double2*>(chunk_in + static_cast<int64_t>(ch + u * stride) * 4);
+      t[2 * u] = rec[0];
+      t[2 * u + 1] = rec[1];
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      a += t[2 * u].x;
+      b += t[2 * u].y;
+      c += t[2 * u + 1].x;
+    }
+  }
+  for (; ch < c1; ch += stride) add_record(chunk_in, ch, a, b, c);
+}
 
 __global__ void __launch_bounds__(kFinalizeThreads)
     finalize_kernel(const __grid_constant__ FinalizeParams fp) {
-  __shared__ double red[(kFinalizeThreads / 32) * 3];
-  double tot_n2 = 0.0, tot_S = 0.0, tot_Q = 0.0;
+  __shared__ double red[kFinalizeWarps * 3];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  grid_dependency_wait();
+  // large shards: the whole CTA, one shard after the other
   for (int s = 0; s < fp.n_shards; ++s) {
     const int c0 = fp.chunk_prefix[s], c1 = fp.chunk_prefix[s + 1];
+    if (c1 - c0 <= kSmallShardChunks) continue;
     double a = 0.0, b = 0.0, c = 0.0;
-    for (int ch = c0 + threadIdx.x; ch < c1; ch += kFinalizeThreads) {
-      const double2* rec =
-          reinterpret_cast<const double2*>(fp.chunk_in + static_cast<int64_t>(ch) * 4);
-      const double2 t0 = rec[0], t1 = rec[1];
-      a += t0.x;
-      b += t0.y;
-      c += t1.x;
-    }
-    block_reduce3<kFinalizeThreads / 32>(a, b, c, red);
+    strided_records(fp.chunk_in, c0, c1, threadIdx.x, kFinalizeThreads, a, b, c);
+    block_reduce3<kFinalizeWarps>(a, b, c, red);
     if (threadIdx.x == 0) {
       double* rec = fp.stats + ABS_STATS_HEADER + s * ABS_SHARD_STRIDE;
       rec[0] = a;
       rec[1] = b;
       rec[2] = c;
       rec[3] = 0.0;
-      tot_n2 += a;
-      tot_S += b;
-      tot_Q += c;
     }
   }
+  // small shards: one warp per shard, round-robin
+  for (int s = warp; s < fp.n_shards; s += kFinalizeWarps) {
+    const int c0 = fp.chunk_prefix[s], c1 = fp.chunk_prefix[s + 1];
+    if (c1 - c0 > kSmallShardChunks) continue;
+    double a = 0.0, b = 0.0, c = 0.0;
+    strided_records(fp.chunk_in, c0, c1, lane, 32, a, b, c);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      a += __shfl_down_sync(0xffffffffu, a, off);
+      b += __shfl_down_sync(0xffffffffu, b, off);
+      c += __shfl_down_sync(0xffffffffu, c, off);
+    }
+    if (lane == 0) {
+      double* rec = fp.stats + ABS_STATS_HEADER + s * ABS_SHARD_STRIDE;
+      rec[0] = a;
+      rec[1] = b;
+      rec[2] = c;
+      rec[3] = 0.0;
+    }
+  }
+  __threadfence_block();
+  __syncthreads();
   if (threadIdx.x == 0) {
+    double tot_n2 = 0.0, tot_S = 0.0, tot_Q = 0.0;
+    for (int s = 0; s < fp.n_shards; ++s) {
+      const volatile double* rec = fp.stats + ABS_STATS_HEADER + s * ABS_SHARD_STRIDE;
+      tot_n2 += rec[0];
+      tot_S += rec[1];
+      tot_Q += rec[2];
+    }
     double T;
     int flags;
     const int64_t b_next = decide_device(tot_S, tot_n2, fp.norm, fp.eta, fp.b_cur, &T, &flags);

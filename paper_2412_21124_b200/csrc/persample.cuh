@@ -35,6 +35,7 @@ template <int VC>
 __global__ void __launch_bounds__(kThreads)
     persample_partial_kernel(const __grid_constant__ PersampleParams prm) {
   const int64_t c0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) * VC;
+  grid_dependency_wait();
   if (c0 >= prm.d) return;
   const int64_t r0 = static_cast<int64_t>(blockIdx.y) * prm.rows_per_block;
   const int64_t r1 = (r0 + prm.rows_per_block < prm.b) ? r0 + prm.rows_per_block : prm.b;
@@ -109,6 +110,7 @@ __global__ void __launch_bounds__(kThreads)
     persample_merge_kernel(const __grid_constant__ PersampleParams prm) {
   __shared__ double red[kWarps * 3];
   const int64_t c = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  grid_dependency_wait();
   double a = 0.0, s = 0.0, q = 0.0;
   if (c < prm.d) {
     double mean = 0.0, m2 = 0.0;
@@ -147,10 +149,33 @@ __global__ void __launch_bounds__(kThreads)
     adamw_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,
                  float* __restrict__ v, int64_t d, const AdamScalars a) {
   const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
+  grid_dependency_wait();
   if (VEC) {
     const int64_t nvec = d >> 2;
-    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < nvec;
-         i += stride) {
+    int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    // two vectors per array in flight per thread
+    for (; i + stride < nvec; i += 2 * stride) {
+      const int64_t j = i + stride;
+      const float4 g0 = __ldcs(reinterpret_cast<const float4*>(g) + i);
+      const float4 g1 = __ldcs(reinterpret_cast<const float4*>(g) + j);
+      float4 p0 = ld_state_16(p + 4 * i), m0 = ld_state_16(m + 4 * i), v0 = ld_state_16(v + 4 * i);
+      float4 p1 = ld_state_16(p + 4 * j), m1 = ld_state_16(m + 4 * j), v1 = ld_state_16(v + 4 * j);
+      adamw_elem(a, g0.x, p0.x, m0.x, v0.x);
+      adamw_elem(a, g0.y, p0.y, m0.y, v0.y);
+      adamw_elem(a, g0.z, p0.z, m0.z, v0.z);
+      adamw_elem(a, g0.w, p0.w, m0.w, v0.w);
+      st_stream_16(p + 4 * i, p0);
+      st_stream_16(m + 4 * i, m0);
+      st_stream_16(v + 4 * i, v0);
+      adamw_elem(a, g1.x, p1.x, m1.x, v1.x);
+      adamw_elem(a, g1.y, p1.y, m1.y, v1.y);
+      adamw_elem(a, g1.z, p1.z, m1.z, v1.z);
+      adamw_elem(a, g1.w, p1.w, m1.w, v1.w);
+      st_stream_16(p + 4 * j, p1);
+      st_stream_16(m + 4 * j, m1);
+      st_stream_16(v + 4 * j, v1);
+    }
+    if (i < nvec) {
       const float4 gg = __ldcs(reinterpret_cast<const float4*>(g) + i);
       float4 pp = ld_state_16(p + 4 * i), mm = ld_state_16(m + 4 * i), vv = ld_state_16(v + 4 * i);
       adamw_elem(a, gg.x, pp.x, mm.x, vv.x);
