@@ -198,9 +198,9 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 
 // tree); shards with few chunks by one warp each.  Thread 0 then adds the shard records
 // in shard order, takes the decision (Algorithm 1: statistic T_k and the If/Else) and
 // writes the header.  The shape of every sum depends only on the chunk counts.
-constexpr int kFinalizeThreads = 256;
+constexpr int kFinalizeThreads = 1024;
 constexpr int kFinalizeWarps = kFinalizeThreads / 32;
-constexpr int kSmallShardChunks = 512;
+constexpr int kSmallShardChunks = 2048;
 
 __device__ __forceinline__ void add_record(const double* chunk_in, int ch, double& a, double& b,
                                            double& c) {
