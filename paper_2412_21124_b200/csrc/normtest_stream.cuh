@@ -202,36 +202,31 @@ constexpr int kFinalizeThreads = 1024;
 constexpr int kFinalizeWarps = kFinalizeThreads / 32;
 constexpr int kSmallShardChunks = 2048;
 
-__device__ __forceinline__ void add_record(const double* chunk_in, int ch, double& a, double& b,
-                                           double& c) {
-  const double2* rec = reinterpret_cast<const double2*>(chunk_in + static_cast<int64_t>(ch) * 4);
-  const double2 t0 = rec[0], t1 = rec[1];
-  a += t0.x;
-  b += t0.y;
-  c += t1.x;
-}
-
-// records c0 + first, c0 + first + stride, ... (< c1), in order, four loads in flight
+// records c0 + first, c0 + first + stride, ... (< c1), added in that order; eight loads in
+// flight per pass (absent records read as +0.0, which leaves the sums unchanged)
 __device__ __forceinline__ void strided_records(const double* chunk_in, int c0, int c1, int first,
                                                 int stride, double& a, double& b, double& c) {
-  int ch = c0 + first;
-  for (; ch + 3 * stride < c1; ch += 4 * stride) {
-    double2 t[8];
+  for (int ch = c0 + first; ch < c1; ch += 8 * stride) {
+    double2 t[16];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const double2* rec =
-          reinterpret_cast<const double2*>(chunk_in + static_cast<int64_t>(ch + u * stride) * 4);
-      t[2 * u] = rec[0];
-      t[2 * u + 1] = rec[1];
+    for (int u = 0; u < 8; ++u) {
+      const int r = ch + u * stride;
+      if (r < c1) {
+        const double2* rec = reinterpret_cast<const double2*>(chunk_in + static_cast<int64_t>(r) * 4);
+        t[2 * u] = rec[0];
+        t[2 * u + 1] = rec[1];
+      } else {
+        t[2 * u] = make_double2(0.0, 0.0);
+        t[2 * u + 1] = make_double2(0.0, 0.0);
+      }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < 8; ++u) {
       a += t[2 * u].x;
       b += t[2 * u].y;
       c += t[2 * u + 1].x;
     }
   }
-  for (; ch < c1; ch += stride) add_record(chunk_in, ch, a, b, c);
 }
 
 __global__ void __launch_bounds__(kFinalizeThreads)
