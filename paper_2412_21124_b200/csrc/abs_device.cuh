@@ -80,6 +80,27 @@ __device__ __forceinline__ void st_stream_16(float* p, float4 x) {
   __stcs(reinterpret_cast<float4*>(p), x);
 }
 
+// 256-bit accesses (sm_100): with bf16 gradients a thread owns 8 consecutive coordinates,
+// i.e. 32 bytes of each fp32 array.  One 256-bit access per array touches whole 32-byte
+// sectors; two 128-bit accesses would each touch half of every sector, doubling the
+// requests the load/store unit and the L2 see (visible as lg_throttle stalls).
+struct alignas(32) Float8 {
+  float4 lo, hi;
+};
+__device__ __forceinline__ Float8 ld_state_32(const float* p) {
+  Float8 r;
+  asm volatile("ld.global.cs.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(r.lo.x), "=f"(r.lo.y), "=f"(r.lo.z), "=f"(r.lo.w), "=f"(r.hi.x),
+                 "=f"(r.hi.y), "=f"(r.hi.z), "=f"(r.hi.w)
+               : "l"(p));
+  return r;
+}
+__device__ __forceinline__ void st_stream_32(float* p, const float4& lo, const float4& hi) {
+  asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(lo.x),
+               "f"(lo.y), "f"(lo.z), "f"(lo.w), "f"(hi.x), "f"(hi.y), "f"(hi.z), "f"(hi.w)
+               : "memory");
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 

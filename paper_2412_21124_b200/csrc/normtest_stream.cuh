@@ -83,6 +83,10 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 
     normtest_stream_kernel(const __grid_constant__ StreamParams prm) {
   constexpr int V = GT::kVec;
   constexpr int NF4 = V / 4; // float4 per thread-row of an fp32 array
+  // 256-bit stores of the fp32 arrays pay off for few workers (K <= 7: +3..9% measured) and
+  // cost about 1% for K >= 8, where the stores of the first half are better issued early;
+  // 256-bit loads never hurt.
+  constexpr bool kWideStores = (V == 8) && (KB < 8 || !EXACT) && KB <= 8;
   __shared__ double red[kWarps * 3];
 
   const int K = EXACT ? KB : prm.K;
@@ -101,20 +105,22 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 
     const int64_t shard_hi = prm.shard_off[lo_s + 1];
     const int64_t hi = (lo + prm.chunk_elems < shard_hi) ? lo + prm.chunk_elems : shard_hi;
 
-    // 16-byte alignment of every stream at this chunk (uniform across the CTA)
-    uintptr_t bits = 0;
+    // alignment of every stream at this chunk (uniform across the CTA): 16 bytes selects
+    // the vector path; 32 bytes of the fp32 arrays additionally selects 256-bit accesses
+    uintptr_t bits = 0, bits_f32 = 0;
 #pragma unroll
     for (int k = 0; k < KB; ++k)
       if (EXACT || k < K)
         bits |= reinterpret_cast<uintptr_t>(prm.grads[k]) +
                 static_cast<uintptr_t>(lo) * sizeof(typename GT::scalar);
-    if (prm.gbar) bits |= reinterpret_cast<uintptr_t>(prm.gbar) + static_cast<uintptr_t>(lo) * 4;
+    if (prm.gbar) bits_f32 |= reinterpret_cast<uintptr_t>(prm.gbar) + static_cast<uintptr_t>(lo) * 4;
     if (ADAM) {
-      bits |= reinterpret_cast<uintptr_t>(prm.p) + static_cast<uintptr_t>(lo) * 4;
-      bits |= reinterpret_cast<uintptr_t>(prm.m) + static_cast<uintptr_t>(lo) * 4;
-      bits |= reinterpret_cast<uintptr_t>(prm.v) + static_cast<uintptr_t>(lo) * 4;
+      bits_f32 |= reinterpret_cast<uintptr_t>(prm.p) + static_cast<uintptr_t>(lo) * 4;
+      bits_f32 |= reinterpret_cast<uintptr_t>(prm.m) + static_cast<uintptr_t>(lo) * 4;
+      bits_f32 |= reinterpret_cast<uintptr_t>(prm.v) + static_cast<uintptr_t>(lo) * 4;
     }
-    const bool aligned = (bits & 15) == 0;
+    const bool aligned = ((bits | bits_f32) & 15) == 0;
+    const bool wide = (V == 8) && (bits_f32 & 31) == 0;
     if (!waited) {  // everything above used kernel parameters only
       grid_dependency_wait();
       waited = true;
@@ -134,14 +140,23 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 
             raw[k] = ld_once_16(reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) + base);
         float4 pw[NF4], pm[NF4], pv[NF4];
         if (ADAM) {
+          if (V == 8 && wide) {
+            const Float8 a = ld_state_32(prm.p + base), b = ld_state_32(prm.m + base),
+                         c = ld_state_32(prm.v + base);
+            pw[0] = a.lo; pw[NF4 - 1] = a.hi;
+            pm[0] = b.lo; pm[NF4 - 1] = b.hi;
+            pv[0] = c.lo; pv[NF4 - 1] = c.hi;
+          } else {
 #pragma unroll
-          for (int q = 0; q < NF4; ++q) {
-            pw[q] = ld_state_16(prm.p + base + 4 * q);
-            pm[q] = ld_state_16(prm.m + base + 4 * q);
-            pv[q] = ld_state_16(prm.v + base + 4 * q);
+            for (int q = 0; q < NF4; ++q) {
+              pw[q] = ld_state_16(prm.p + base + 4 * q);
+              pm[q] = ld_state_16(prm.m + base + 4 * q);
+              pv[q] = ld_state_16(prm.v + base + 4 * q);
+            }
           }
         }
         // four coordinates at a time, stored as soon as they are done (short live ranges)
+        float4 gb_lo = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int q = 0; q < NF4; ++q) {
           float gb[4];
@@ -162,12 +177,27 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 
             row_Q += sq;
             if (ADAM) adamw_elem(prm.adam, mean, w4[j], m4[j], v4[j]);
           }
-          if (prm.gbar)
-            st_stream_16(prm.gbar + base + 4 * q, make_float4(gb[0], gb[1], gb[2], gb[3]));
-          if (ADAM) {
-            st_stream_16(prm.p + base + 4 * q, pw[q]);
-            st_stream_16(prm.m + base + 4 * q, pm[q]);
-            st_stream_16(prm.v + base + 4 * q, pv[q]);
+          if (kWideStores && wide) {
+            // hold the first half back; store all 32 bytes with the second half
+            if (q == 0) {
+              gb_lo = make_float4(gb[0], gb[1], gb[2], gb[3]);
+            } else {
+              if (prm.gbar)
+                st_stream_32(prm.gbar + base, gb_lo, make_float4(gb[0], gb[1], gb[2], gb[3]));
+              if (ADAM) {
+                st_stream_32(prm.p + base, pw[0], pw[NF4 - 1]);
+                st_stream_32(prm.m + base, pm[0], pm[NF4 - 1]);
+                st_stream_32(prm.v + base, pv[0], pv[NF4 - 1]);
+              }
+            }
+          } else {
+            if (prm.gbar)
+              st_stream_16(prm.gbar + base + 4 * q, make_float4(gb[0], gb[1], gb[2], gb[3]));
+            if (ADAM) {
+              st_stream_16(prm.p + base + 4 * q, pw[q]);
+              st_stream_16(prm.m + base + 4 * q, pm[q]);
+              st_stream_16(prm.v + base + 4 * q, pv[q]);
+            }
           }
         }
       } else if (base < hi) {
