@@ -78,148 +78,174 @@ __device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t 
   sums[2] = row_Q;
 }
 
+// Where a chunk lies and how its streams are aligned (uniform across the CTA; computed
+// from kernel parameters only).
+struct ChunkGeometry {
+  int64_t lo, hi;  // coordinates [lo, hi)
+  bool aligned;    // every stream 16-byte aligned at lo: vector path
+  bool wide;       // fp32 arrays also 32-byte aligned: 256-bit accesses (bf16 gradients)
+};
+
+template <typename GT, int KB, bool EXACT, bool ADAM>
+__device__ __forceinline__ ChunkGeometry chunk_geometry(const StreamParams& prm, int K, int chunk) {
+  // shard that owns this chunk: largest s with chunk_prefix[s] <= chunk
+  int lo_s = 0, hi_s = prm.n_shards;
+  while (hi_s - lo_s > 1) {
+    const int mid = (lo_s + hi_s) >> 1;
+    if (prm.chunk_prefix[mid] <= chunk) lo_s = mid; else hi_s = mid;
+  }
+  ChunkGeometry g;
+  g.lo = prm.shard_off[lo_s] +
+         static_cast<int64_t>(chunk - prm.chunk_prefix[lo_s]) * prm.chunk_elems;
+  const int64_t shard_hi = prm.shard_off[lo_s + 1];
+  g.hi = (g.lo + prm.chunk_elems < shard_hi) ? g.lo + prm.chunk_elems : shard_hi;
+  uintptr_t bits = 0, bits_f32 = 0;
+#pragma unroll
+  for (int k = 0; k < KB; ++k)
+    if (EXACT || k < K)
+      bits |= reinterpret_cast<uintptr_t>(prm.grads[k]) +
+              static_cast<uintptr_t>(g.lo) * sizeof(typename GT::scalar);
+  if (prm.gbar) bits_f32 |= reinterpret_cast<uintptr_t>(prm.gbar) + static_cast<uintptr_t>(g.lo) * 4;
+  if (ADAM) {
+    bits_f32 |= reinterpret_cast<uintptr_t>(prm.p) + static_cast<uintptr_t>(g.lo) * 4;
+    bits_f32 |= reinterpret_cast<uintptr_t>(prm.m) + static_cast<uintptr_t>(g.lo) * 4;
+    bits_f32 |= reinterpret_cast<uintptr_t>(prm.v) + static_cast<uintptr_t>(g.lo) * 4;
+  }
+  g.aligned = ((bits | bits_f32) & 15) == 0;
+  g.wide = (GT::kVec == 8) && (bits_f32 & 31) == 0;
+  return g;
+}
+
+// Register-direct processing of one chunk: every thread-row is loaded with 128/256-bit
+// global loads straight into registers.  Adds this thread's sums to acc_*.
 template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
-__global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 ? 2 : 1)))
-    normtest_stream_kernel(const __grid_constant__ StreamParams prm) {
+__device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K,
+                                                  const ChunkGeometry& cg, double& acc_n2,
+                                                  double& acc_S, double& acc_Q) {
   constexpr int V = GT::kVec;
   constexpr int NF4 = V / 4; // float4 per thread-row of an fp32 array
   // 256-bit stores of the fp32 arrays pay off for few workers (K <= 7: +3..9% measured) and
   // cost about 1% for K >= 8, where the stores of the first half are better issued early;
   // 256-bit loads never hurt.
   constexpr bool kWideStores = (V == 8) && (KB < 8 || !EXACT) && KB <= 8;
-  __shared__ double red[kWarps * 3];
-
-  const int K = EXACT ? KB : prm.K;
   const int tid = threadIdx.x;
-  bool waited = false;
+  const int64_t hi = cg.hi;
+  const bool wide = cg.wide;
 
-  for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
-    // shard that owns this chunk: largest s with chunk_prefix[s] <= chunk
-    int lo_s = 0, hi_s = prm.n_shards;
-    while (hi_s - lo_s > 1) {
-      const int mid = (lo_s + hi_s) >> 1;
-      if (prm.chunk_prefix[mid] <= chunk) lo_s = mid; else hi_s = mid;
-    }
-    const int64_t lo = prm.shard_off[lo_s] +
-                       static_cast<int64_t>(chunk - prm.chunk_prefix[lo_s]) * prm.chunk_elems;
-    const int64_t shard_hi = prm.shard_off[lo_s + 1];
-    const int64_t hi = (lo + prm.chunk_elems < shard_hi) ? lo + prm.chunk_elems : shard_hi;
+  for (int64_t row_lo = cg.lo; row_lo < hi; row_lo += kThreads * V) {
+    const int64_t base = row_lo + static_cast<int64_t>(tid) * V;
+    float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
 
-    // alignment of every stream at this chunk (uniform across the CTA): 16 bytes selects
-    // the vector path; 32 bytes of the fp32 arrays additionally selects 256-bit accesses
-    uintptr_t bits = 0, bits_f32 = 0;
+    if (cg.aligned && (row_lo + kThreads * V <= hi)) {
+      uint4 raw[KB];
 #pragma unroll
-    for (int k = 0; k < KB; ++k)
-      if (EXACT || k < K)
-        bits |= reinterpret_cast<uintptr_t>(prm.grads[k]) +
-                static_cast<uintptr_t>(lo) * sizeof(typename GT::scalar);
-    if (prm.gbar) bits_f32 |= reinterpret_cast<uintptr_t>(prm.gbar) + static_cast<uintptr_t>(lo) * 4;
-    if (ADAM) {
-      bits_f32 |= reinterpret_cast<uintptr_t>(prm.p) + static_cast<uintptr_t>(lo) * 4;
-      bits_f32 |= reinterpret_cast<uintptr_t>(prm.m) + static_cast<uintptr_t>(lo) * 4;
-      bits_f32 |= reinterpret_cast<uintptr_t>(prm.v) + static_cast<uintptr_t>(lo) * 4;
+      for (int k = 0; k < KB; ++k)
+        if (EXACT || k < K)
+          raw[k] = ld_once_16(reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) + base);
+      float4 pw[NF4], pm[NF4], pv[NF4];
+      if (ADAM) {
+        if (V == 8 && wide) {
+          const Float8 a = ld_state_32(prm.p + base), b = ld_state_32(prm.m + base),
+                       c = ld_state_32(prm.v + base);
+          pw[0] = a.lo; pw[NF4 - 1] = a.hi;
+          pm[0] = b.lo; pm[NF4 - 1] = b.hi;
+          pv[0] = c.lo; pv[NF4 - 1] = c.hi;
+        } else {
+#pragma unroll
+          for (int q = 0; q < NF4; ++q) {
+            pw[q] = ld_state_16(prm.p + base + 4 * q);
+            pm[q] = ld_state_16(prm.m + base + 4 * q);
+            pv[q] = ld_state_16(prm.v + base + 4 * q);
+          }
+        }
+      }
+      // four coordinates at a time, stored as soon as they are done (short live ranges)
+      float4 gb_lo = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int q = 0; q < NF4; ++q) {
+        float gb[4];
+        float* w4 = reinterpret_cast<float*>(&pw[q]);
+        float* m4 = reinterpret_cast<float*>(&pm[q]);
+        float* v4 = reinterpret_cast<float*>(&pv[q]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float g[KB];
+#pragma unroll
+          for (int k = 0; k < KB; ++k)
+            g[k] = (EXACT || k < K) ? GT::elem(raw[k], 4 * q + j) : 0.f;
+          float dev2, sq;
+          const float mean = coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
+          gb[j] = mean;
+          row_n2 = fmaf(mean, mean, row_n2);
+          row_S += dev2;
+          row_Q += sq;
+          if (ADAM) adamw_elem(prm.adam, mean, w4[j], m4[j], v4[j]);
+        }
+        if (kWideStores && wide) {
+          // hold the first half back; store all 32 bytes with the second half
+          if (q == 0) {
+            gb_lo = make_float4(gb[0], gb[1], gb[2], gb[3]);
+          } else {
+            if (prm.gbar)
+              st_stream_32(prm.gbar + base, gb_lo, make_float4(gb[0], gb[1], gb[2], gb[3]));
+            if (ADAM) {
+              st_stream_32(prm.p + base, pw[0], pw[NF4 - 1]);
+              st_stream_32(prm.m + base, pm[0], pm[NF4 - 1]);
+              st_stream_32(prm.v + base, pv[0], pv[NF4 - 1]);
+            }
+          }
+        } else {
+          if (prm.gbar)
+            st_stream_16(prm.gbar + base + 4 * q, make_float4(gb[0], gb[1], gb[2], gb[3]));
+          if (ADAM) {
+            st_stream_16(prm.p + base + 4 * q, pw[q]);
+            st_stream_16(prm.m + base + 4 * q, pm[q]);
+            st_stream_16(prm.v + base + 4 * q, pv[q]);
+          }
+        }
+      }
+    } else if (base < hi) {
+      float sums[3];
+      scalar_row<GT, KB, EXACT, ADAM, WITHQ>(prm, K, base, hi, sums);
+      row_n2 = sums[0];
+      row_S = sums[1];
+      row_Q = sums[2];
     }
-    const bool aligned = ((bits | bits_f32) & 15) == 0;
-    const bool wide = (V == 8) && (bits_f32 & 31) == 0;
+    acc_n2 += static_cast<double>(row_n2);
+    acc_S += static_cast<double>(row_S);
+    if (WITHQ) acc_Q += static_cast<double>(row_Q);
+  }
+}
+
+// CTA-wide fixed-order reduction of the per-thread sums and the chunk record.
+template <bool WITHQ>
+__device__ __forceinline__ void write_chunk_record(const StreamParams& prm, int chunk, double acc_n2,
+                                                   double acc_S, double acc_Q, double* red) {
+  block_reduce3<kWarps>(acc_n2, acc_S, acc_Q, red);
+  if (threadIdx.x == 0) {
+    double* out = prm.chunk_out + static_cast<int64_t>(chunk) * 4;
+    out[0] = acc_n2;
+    out[1] = acc_S;
+    out[2] = WITHQ ? acc_Q : __longlong_as_double(0x7ff8000000000000ll);  // NaN: not computed
+    out[3] = 0.0;
+  }
+}
+
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+__global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 ? 2 : 1)))
+    normtest_stream_kernel(const __grid_constant__ StreamParams prm) {
+  __shared__ double red[kWarps * 3];
+  const int K = EXACT ? KB : prm.K;
+  bool waited = false;
+  for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
+    const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, K, chunk);
     if (!waited) {  // everything above used kernel parameters only
       grid_dependency_wait();
       waited = true;
     }
-
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
-
-    for (int64_t row_lo = lo; row_lo < hi; row_lo += kThreads * V) {
-      const int64_t base = row_lo + static_cast<int64_t>(tid) * V;
-      float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
-
-      if (aligned && (row_lo + kThreads * V <= hi)) {
-        uint4 raw[KB];
-#pragma unroll
-        for (int k = 0; k < KB; ++k)
-          if (EXACT || k < K)
-            raw[k] = ld_once_16(reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) + base);
-        float4 pw[NF4], pm[NF4], pv[NF4];
-        if (ADAM) {
-          if (V == 8 && wide) {
-            const Float8 a = ld_state_32(prm.p + base), b = ld_state_32(prm.m + base),
-                         c = ld_state_32(prm.v + base);
-            pw[0] = a.lo; pw[NF4 - 1] = a.hi;
-            pm[0] = b.lo; pm[NF4 - 1] = b.hi;
-            pv[0] = c.lo; pv[NF4 - 1] = c.hi;
-          } else {
-#pragma unroll
-            for (int q = 0; q < NF4; ++q) {
-              pw[q] = ld_state_16(prm.p + base + 4 * q);
-              pm[q] = ld_state_16(prm.m + base + 4 * q);
-              pv[q] = ld_state_16(prm.v + base + 4 * q);
-            }
-          }
-        }
-        // four coordinates at a time, stored as soon as they are done (short live ranges)
-        float4 gb_lo = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int q = 0; q < NF4; ++q) {
-          float gb[4];
-          float* w4 = reinterpret_cast<float*>(&pw[q]);
-          float* m4 = reinterpret_cast<float*>(&pm[q]);
-          float* v4 = reinterpret_cast<float*>(&pv[q]);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float g[KB];
-#pragma unroll
-            for (int k = 0; k < KB; ++k)
-              g[k] = (EXACT || k < K) ? GT::elem(raw[k], 4 * q + j) : 0.f;
-            float dev2, sq;
-            const float mean = coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
-            gb[j] = mean;
-            row_n2 = fmaf(mean, mean, row_n2);
-            row_S += dev2;
-            row_Q += sq;
-            if (ADAM) adamw_elem(prm.adam, mean, w4[j], m4[j], v4[j]);
-          }
-          if (kWideStores && wide) {
-            // hold the first half back; store all 32 bytes with the second half
-            if (q == 0) {
-              gb_lo = make_float4(gb[0], gb[1], gb[2], gb[3]);
-            } else {
-              if (prm.gbar)
-                st_stream_32(prm.gbar + base, gb_lo, make_float4(gb[0], gb[1], gb[2], gb[3]));
-              if (ADAM) {
-                st_stream_32(prm.p + base, pw[0], pw[NF4 - 1]);
-                st_stream_32(prm.m + base, pm[0], pm[NF4 - 1]);
-                st_stream_32(prm.v + base, pv[0], pv[NF4 - 1]);
-              }
-            }
-          } else {
-            if (prm.gbar)
-              st_stream_16(prm.gbar + base + 4 * q, make_float4(gb[0], gb[1], gb[2], gb[3]));
-            if (ADAM) {
-              st_stream_16(prm.p + base + 4 * q, pw[q]);
-              st_stream_16(prm.m + base + 4 * q, pm[q]);
-              st_stream_16(prm.v + base + 4 * q, pv[q]);
-            }
-          }
-        }
-      } else if (base < hi) {
-        float sums[3];
-        scalar_row<GT, KB, EXACT, ADAM, WITHQ>(prm, K, base, hi, sums);
-        row_n2 = sums[0];
-        row_S = sums[1];
-        row_Q = sums[2];
-      }
-      acc_n2 += static_cast<double>(row_n2);
-      acc_S += static_cast<double>(row_S);
-      if (WITHQ) acc_Q += static_cast<double>(row_Q);
-    }
-
-    block_reduce3<kWarps>(acc_n2, acc_S, acc_Q, red);
-    if (tid == 0) {
-      double* out = prm.chunk_out + static_cast<int64_t>(chunk) * 4;
-      out[0] = acc_n2;
-      out[1] = acc_S;
-      out[2] = WITHQ ? acc_Q : __longlong_as_double(0x7ff8000000000000ll);  // NaN: not computed
-      out[3] = 0.0;
-    }
+    chunk_rows_direct<GT, KB, EXACT, ADAM, WITHQ>(prm, K, cg, acc_n2, acc_S, acc_Q);
+    write_chunk_record<WITHQ>(prm, chunk, acc_n2, acc_S, acc_Q, red);
   }
 }
 
