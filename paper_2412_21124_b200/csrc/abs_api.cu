@@ -8,6 +8,7 @@
 #include <utility>
 
 #include "abs_device.cuh"
+#include "normtest_bulk.cuh"
 #include "normtest_stream.cuh"
 #include "persample.cuh"
 
@@ -109,28 +110,59 @@ int make_layout(int64_t d, const int64_t* shard_offsets, int n_shards, Layout* L
   return ABS_OK;
 }
 
+// Launch with dynamic shared memory above the 48 KB default.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                            cudaStream_t st, Args&&... args) {
+  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel),
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+// One (dtype, K bucket) instantiation: the bulk-async kernel where its stages fit two CTAs
+// per SM, else the register-direct kernel.
+template <typename GT, int KB, bool EXACT, bool ADAM>
+cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
+  const dim3 grid(static_cast<unsigned>(prm.n_chunks)), block(kThreads);
+  if constexpr (bulk_fits<GT, KB, ADAM>()) {
+    constexpr size_t smem = static_cast<size_t>(kBulkStages) * bulk_stage_bytes<GT, KB, ADAM>();
+    return launch_pdl_smem(normtest_bulk_kernel<GT, KB, EXACT, ADAM, !ADAM>, grid, block, smem, st,
+                           prm);
+  } else {
+    return launch_pdl(normtest_stream_kernel<GT, KB, EXACT, ADAM, !ADAM>, grid, block, st, prm);
+  }
+}
+
 // The fused kernel leaves Q out (its stats slot reads NaN): at the power cap the K extra
 // multiply-adds per coordinate cost about 1% of bandwidth.  The unfused test computes it.
 template <typename GT, bool ADAM>
 cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
-  const int grid = prm.n_chunks;
   const int K = prm.K;
-#define ABS_LAUNCH(KB, EXACT) \
-  launch_pdl(normtest_stream_kernel<GT, KB, EXACT, ADAM, !ADAM>, dim3(grid), dim3(kThreads), st, prm)
   switch (K) {
-    case 1: return ABS_LAUNCH(1, true);
-    case 2: return ABS_LAUNCH(2, true);
-    case 3: return ABS_LAUNCH(3, true);
-    case 4: return ABS_LAUNCH(4, true);
-    case 8: return ABS_LAUNCH(8, true);
-    case 16: return ABS_LAUNCH(16, true);
-    case 32: return ABS_LAUNCH(32, true);
+    case 1: return launch_one<GT, 1, true, ADAM>(prm, st);
+    case 2: return launch_one<GT, 2, true, ADAM>(prm, st);
+    case 3: return launch_one<GT, 3, true, ADAM>(prm, st);
+    case 4: return launch_one<GT, 4, true, ADAM>(prm, st);
+    case 8: return launch_one<GT, 8, true, ADAM>(prm, st);
+    case 16: return launch_one<GT, 16, true, ADAM>(prm, st);
+    case 32: return launch_one<GT, 32, true, ADAM>(prm, st);
     default:
-      if (K < 8) return ABS_LAUNCH(8, false);
-      if (K < 16) return ABS_LAUNCH(16, false);
-      return ABS_LAUNCH(32, false);
+      if (K < 8) return launch_one<GT, 8, false, ADAM>(prm, st);
+      if (K < 16) return launch_one<GT, 16, false, ADAM>(prm, st);
+      return launch_one<GT, 32, false, ADAM>(prm, st);
   }
-#undef ABS_LAUNCH
 }
 
 int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
