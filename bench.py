@@ -306,7 +306,7 @@ def run_ours(args, d):
     roofline = {"bound": "hbm", "achieved": kernel_gbs, "peak": peak, "unit": "GB/s",
                 "frac": kernel_gbs / peak, "peak_source": peak_src,
                 "frac_of_nominal_8TBs": kernel_gbs / NOMINAL_HBM_GBS,
-                "kernel": "normtest_stream_kernel<bf16,K=8,fused AdamW> (+ finalize, same timed call)",
+                "kernel": "normtest_bulk_kernel<bf16,K=8,fused AdamW> (cp.async.bulk staging; + finalize, same timed call)",
                 "algorithmic_bytes_per_launch": bytes_step,
                 "traffic": recorded_traffic(d)}
     cpu = None
