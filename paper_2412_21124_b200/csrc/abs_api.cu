@@ -131,17 +131,22 @@ cudaError_t launch_pdl_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
-// One (dtype, K bucket) instantiation: the bulk-async kernel where its stages fit two CTAs
-// per SM, else the register-direct kernel.
+// One (dtype, K bucket) instantiation: the bulk-async kernel where its stages leave room for
+// two or three CTAs per SM, else the register-direct kernel.
 template <typename GT, int KB, bool EXACT, bool ADAM>
 cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
-  const dim3 grid(static_cast<unsigned>(prm.n_chunks)), block(kThreads);
-  if constexpr (bulk_fits<GT, KB, ADAM>()) {
-    constexpr size_t smem = static_cast<size_t>(kBulkStages) * bulk_stage_bytes<GT, KB, ADAM>();
-    return launch_pdl_smem(normtest_bulk_kernel<GT, KB, EXACT, ADAM, !ADAM>, grid, block, smem, st,
-                           prm);
+  const dim3 grid(static_cast<unsigned>(prm.n_chunks));
+  // (the 512-coordinate tile loses to the register-direct kernel for the predicated
+  // K buckets, measured at K=12)
+  constexpr int tile = (bulk_tile<GT, KB, ADAM>() == 512 && !EXACT) ? 0 : bulk_tile<GT, KB, ADAM>();
+  if constexpr (tile > 0) {
+    constexpr size_t smem =
+        static_cast<size_t>(kBulkStages) * bulk_stage_bytes<GT, KB, ADAM>(tile);
+    return launch_pdl_smem(normtest_bulk_kernel<GT, KB, EXACT, ADAM, !ADAM, tile>, grid,
+                           dim3(tile / 4), smem, st, prm);
   } else {
-    return launch_pdl(normtest_stream_kernel<GT, KB, EXACT, ADAM, !ADAM>, grid, block, st, prm);
+    return launch_pdl(normtest_stream_kernel<GT, KB, EXACT, ADAM, !ADAM>, grid, dim3(kThreads), st,
+                      prm);
   }
 }
 

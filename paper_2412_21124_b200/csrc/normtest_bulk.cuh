@@ -24,19 +24,24 @@
 
 namespace absnt {
 
-constexpr int kBulkTile = 1024;          // coordinates per stage = 4 per thread
 constexpr int kBulkStages = 3;
 constexpr int kBulkWaitLimit = 1 << 22;  // mbarrier polls before giving up
+constexpr int kSmemPerSM = 224 * 1024;   // budget for dynamic shared memory per SM
 
-// bytes of one stage
+// bytes of one stage of `tile` coordinates
 template <typename GT, int KB, bool ADAM>
-__host__ __device__ constexpr int bulk_stage_bytes() {
-  return kBulkTile * (KB * static_cast<int>(sizeof(typename GT::scalar)) + (ADAM ? 12 : 0) + 4);
+__host__ __device__ constexpr int bulk_stage_bytes(int tile) {
+  return tile * (KB * static_cast<int>(sizeof(typename GT::scalar)) + (ADAM ? 12 : 0) + 4);
 }
-// the bulk kernel is offered where three stages of two CTAs fit one SM's shared memory
+// Tile size (coordinates per stage, 4 per thread): 1024 with two 256-thread CTAs per SM
+// where three stages of both fit; else 512 with three 128-thread CTAs per SM; else 0 (the
+// register-direct kernel is used).  With a single resident CTA the staging loses to the
+// register-direct kernel, so those shapes are not offered.
 template <typename GT, int KB, bool ADAM>
-__host__ __device__ constexpr bool bulk_fits() {
-  return kBulkStages * bulk_stage_bytes<GT, KB, ADAM>() <= 112 * 1024;
+__host__ __device__ constexpr int bulk_tile() {
+  return 2 * kBulkStages * bulk_stage_bytes<GT, KB, ADAM>(1024) <= kSmemPerSM
+             ? 1024
+             : (3 * kBulkStages * bulk_stage_bytes<GT, KB, ADAM>(512) <= kSmemPerSM ? 512 : 0);
 }
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {
@@ -119,18 +124,20 @@ struct BulkGrad<F32> {
   }
 };
 
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
-__global__ void __launch_bounds__(kThreads, 2)
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ, int TILE>
+__global__ void __launch_bounds__(TILE / 4, (TILE == 1024 ? 2 : 3))
     normtest_bulk_kernel(const __grid_constant__ StreamParams prm) {
+  constexpr int kBulkTile = TILE;
+  constexpr int NT = TILE / 4;  // threads
   constexpr int GB = kBulkTile * static_cast<int>(sizeof(typename GT::scalar));  // gradient segment
   constexpr int FB = kBulkTile * 4;                                              // fp32 segment
   constexpr int OFF_P = KB * GB, OFF_M = OFF_P + (ADAM ? FB : 0), OFF_V = OFF_M + (ADAM ? FB : 0);
   constexpr int OFF_GBAR = OFF_V + (ADAM ? FB : 0);
   constexpr int STAGE = OFF_GBAR + FB;
-  static_assert(STAGE == bulk_stage_bytes<GT, KB, ADAM>(), "stage layout");
+  static_assert(STAGE == bulk_stage_bytes<GT, KB, ADAM>(TILE), "stage layout");
   extern __shared__ __align__(128) unsigned char stages[];
   __shared__ uint64_t full[kBulkStages];
-  __shared__ double red[kWarps * 3];
+  __shared__ double red[(NT / 32) * 3];
 
   const int K = EXACT ? KB : prm.K;
   const int tid = threadIdx.x;
@@ -155,7 +162,7 @@ __global__ void __launch_bounds__(kThreads, 2)
     const bool bulk = cg.aligned && (cg.hi - cg.lo == prm.chunk_elems) &&
                       (prm.chunk_elems % kBulkTile == 0);
     if (!bulk) {
-      chunk_rows_direct<GT, KB, EXACT, ADAM, WITHQ>(prm, K, cg, acc_n2, acc_S, acc_Q);
+      chunk_rows_direct<GT, KB, EXACT, ADAM, WITHQ, NT>(prm, K, cg, acc_n2, acc_S, acc_Q);
     } else {
       const int n_tiles = prm.chunk_elems / kBulkTile;
       const uint32_t tx_bytes = static_cast<uint32_t>(K * GB + (ADAM ? 3 * FB : 0));
@@ -249,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 2)
       if (tid == 0) bulk_wait_stores_read();
     }
     if (lost) acc_S = __longlong_as_double(0x7ff8000000000000ll);  // poison: a copy was lost
-    write_chunk_record<WITHQ>(prm, chunk, acc_n2, acc_S, acc_Q, red);
+    write_chunk_record<WITHQ, NT>(prm, chunk, acc_n2, acc_S, acc_Q, red);
   }
   if (tid == 0) {
     bulk_wait_stores_done();

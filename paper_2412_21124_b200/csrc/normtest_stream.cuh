@@ -118,7 +118,7 @@ __device__ __forceinline__ ChunkGeometry chunk_geometry(const StreamParams& prm,
 
 // Register-direct processing of one chunk: every thread-row is loaded with 128/256-bit
 // global loads straight into registers.  Adds this thread's sums to acc_*.
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ, int NT = kThreads>
 __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K,
                                                   const ChunkGeometry& cg, double& acc_n2,
                                                   double& acc_S, double& acc_Q) {
@@ -132,11 +132,11 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
   const int64_t hi = cg.hi;
   const bool wide = cg.wide;
 
-  for (int64_t row_lo = cg.lo; row_lo < hi; row_lo += kThreads * V) {
+  for (int64_t row_lo = cg.lo; row_lo < hi; row_lo += NT * V) {
     const int64_t base = row_lo + static_cast<int64_t>(tid) * V;
     float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
 
-    if (cg.aligned && (row_lo + kThreads * V <= hi)) {
+    if (cg.aligned && (row_lo + NT * V <= hi)) {
       uint4 raw[KB];
 #pragma unroll
       for (int k = 0; k < KB; ++k)
@@ -218,10 +218,10 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
 }
 
 // CTA-wide fixed-order reduction of the per-thread sums and the chunk record.
-template <bool WITHQ>
+template <bool WITHQ, int NT = kThreads>
 __device__ __forceinline__ void write_chunk_record(const StreamParams& prm, int chunk, double acc_n2,
                                                    double acc_S, double acc_Q, double* red) {
-  block_reduce3<kWarps>(acc_n2, acc_S, acc_Q, red);
+  block_reduce3<NT / 32>(acc_n2, acc_S, acc_Q, red);
   if (threadIdx.x == 0) {
     double* out = prm.chunk_out + static_cast<int64_t>(chunk) * 4;
     out[0] = acc_n2;
