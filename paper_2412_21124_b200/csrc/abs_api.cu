@@ -136,9 +136,12 @@ cudaError_t launch_pdl_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
 template <typename GT, int KB, bool EXACT, bool ADAM>
 cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
   const dim3 grid(static_cast<unsigned>(prm.n_chunks));
-  // (the 512-coordinate tile loses to the register-direct kernel for the predicated
-  // K buckets, measured at K=12)
-  constexpr int tile = (bulk_tile<GT, KB, ADAM>() == 512 && !EXACT) ? 0 : bulk_tile<GT, KB, ADAM>();
+  // Measured exceptions: the 512-coordinate tile loses to the register-direct kernel for the
+  // predicated K buckets (K=12: 5.46 vs 5.80 TB/s), and the unfused test -- 20 B per
+  // coordinate at K=8 bf16, i.e. twice the coordinates per second -- is bound by instruction
+  // issue, where the per-tile bookkeeping of the staged kernel costs 10% (5.95 vs 6.60 TB/s).
+  constexpr int tile =
+      (!ADAM || (bulk_tile<GT, KB, ADAM>() == 512 && !EXACT)) ? 0 : bulk_tile<GT, KB, ADAM>();
   if constexpr (tile > 0) {
     constexpr size_t smem =
         static_cast<size_t>(kBulkStages) * bulk_stage_bytes<GT, KB, ADAM>(tile);
