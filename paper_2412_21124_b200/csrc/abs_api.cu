@@ -268,7 +268,7 @@ size_t abs_persample_stats_bytes(int64_t b, int64_t d) {
   if (b < 2 || d < 1) return 0;
   const int rpb = persample_rows_per_block(b);
   const int64_t nrb = (b + rpb - 1) / rpb;
-  const int64_t n_chunks = (d + kThreads - 1) / kThreads;
+  const int64_t n_chunks = (d + kPsThreads - 1) / kPsThreads;
   return sizeof(double) *
          (ABS_STATS_HEADER + ABS_SHARD_STRIDE + static_cast<size_t>(n_chunks) * 4 +
           3 * static_cast<size_t>(nrb) * static_cast<size_t>(d));
@@ -325,7 +325,7 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
   if (misaligned(G, 4) || misaligned(gbar_out, 4) || misaligned(stats_out, 16) ||
       misaligned(b_next_out, 8))
     return ABS_ERR_ALIGN;
-  const int64_t n_chunks64 = (d + kThreads - 1) / kThreads;
+  const int64_t n_chunks64 = (d + kPsThreads - 1) / kPsThreads;
   const int rpb = persample_rows_per_block(b);
   const int64_t nrb = (b + rpb - 1) / rpb;
   if (n_chunks64 > INT32_MAX || nrb > 65535) return ABS_ERR_RANGE;
@@ -350,15 +350,15 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
   cudaError_t e;
   if (vec) {
     const int64_t cols = (d + 3) / 4;
-    dim3 grid(static_cast<unsigned>((cols + kThreads - 1) / kThreads),
+    dim3 grid(static_cast<unsigned>((cols + kPsThreads - 1) / kPsThreads),
               static_cast<unsigned>(nrb));
-    e = launch_pdl(persample_partial_kernel<4>, grid, dim3(kThreads), st, prm);
+    e = launch_pdl(persample_partial_kernel<4>, grid, dim3(kPsThreads), st, prm);
   } else {
     dim3 grid(static_cast<unsigned>(n_chunks64), static_cast<unsigned>(nrb));
-    e = launch_pdl(persample_partial_kernel<1>, grid, dim3(kThreads), st, prm);
+    e = launch_pdl(persample_partial_kernel<1>, grid, dim3(kPsThreads), st, prm);
   }
   if (e != cudaSuccess) return cuda_fail(e);
-  e = launch_pdl(persample_merge_kernel, dim3(static_cast<unsigned>(n_chunks64)), dim3(kThreads),
+  e = launch_pdl(persample_merge_kernel, dim3(static_cast<unsigned>(n_chunks64)), dim3(kPsThreads),
                  st, prm);
   if (e != cudaSuccess) return cuda_fail(e);
 

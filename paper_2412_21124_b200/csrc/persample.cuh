@@ -9,7 +9,7 @@
 //     delta = mu_g - mean;  mean += delta*n_g/(n+n_g);  M2 += M2_g + delta^2*n*n_g/(n+n_g)
 // (law of total variance).  It writes {mean, M2, Q} per (row block, column).
 // Pass 2 (one thread per column): merges the row blocks in index order with the same
-// update, writes gbar, and reduces {gbar^2, M2, Q} over 256-column chunks for the
+// update, writes gbar, and reduces {gbar^2, M2, Q} over 128-column chunks for the
 // shared finalize kernel.
 // Also here: the stand-alone AdamW kernel.
 #pragma once
@@ -17,7 +17,8 @@
 
 namespace absnt {
 
-constexpr int kGroup = 16; // rows held in registers at a time
+constexpr int kGroup = 16;      // rows held in registers at a time
+constexpr int kPsThreads = 128; // threads per CTA of the per-sample kernels
 
 struct PersampleParams {
   const float* G;
@@ -28,13 +29,13 @@ struct PersampleParams {
   double* ws_m2;
   double* ws_q;
   float* gbar;
-  double* chunk_out; // 4 doubles per 256-column chunk
+  double* chunk_out; // 4 doubles per kPsThreads-column chunk
 };
 
 template <int VC>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kPsThreads, 3)
     persample_partial_kernel(const __grid_constant__ PersampleParams prm) {
-  const int64_t c0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) * VC;
+  const int64_t c0 = (static_cast<int64_t>(blockIdx.x) * kPsThreads + threadIdx.x) * VC;
   grid_dependency_wait();
   if (c0 >= prm.d) return;
   const int64_t r0 = static_cast<int64_t>(blockIdx.y) * prm.rows_per_block;
@@ -106,34 +107,49 @@ __global__ void __launch_bounds__(kThreads)
   }
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kPsThreads)
     persample_merge_kernel(const __grid_constant__ PersampleParams prm) {
-  __shared__ double red[kWarps * 3];
-  const int64_t c = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+  __shared__ double red[(kPsThreads / 32) * 3];
+  const int64_t c = static_cast<int64_t>(blockIdx.x) * kPsThreads + threadIdx.x;
   grid_dependency_wait();
   double a = 0.0, s = 0.0, q = 0.0;
   if (c < prm.d) {
     double mean = 0.0, m2 = 0.0;
     int64_t n = 0;
-    for (int rb = 0; rb < prm.n_row_blocks; ++rb) {
-      const int64_t r0 = static_cast<int64_t>(rb) * prm.rows_per_block;
-      const int64_t nb = (r0 + prm.rows_per_block < prm.b) ? prm.rows_per_block : prm.b - r0;
-      const double mu = prm.ws_mean[static_cast<int64_t>(rb) * prm.d + c];
-      const double nn = static_cast<double>(n + nb);
-      const double w_mean = static_cast<double>(nb) / nn;
-      const double delta = mu - mean;
-      mean += delta * w_mean;
-      m2 += prm.ws_m2[static_cast<int64_t>(rb) * prm.d + c] +
-            delta * delta * (static_cast<double>(n) * w_mean);
-      q += prm.ws_q[static_cast<int64_t>(rb) * prm.d + c];
-      n += nb;
+    // row blocks in index order, eight records in flight at a time
+    for (int rb0 = 0; rb0 < prm.n_row_blocks; rb0 += 8) {
+      double mu[8], mm[8], qq[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int rb = rb0 + u;
+        const bool in = rb < prm.n_row_blocks;
+        const int64_t o = static_cast<int64_t>(in ? rb : 0) * prm.d + c;
+        mu[u] = in ? prm.ws_mean[o] : 0.0;
+        mm[u] = in ? prm.ws_m2[o] : 0.0;
+        qq[u] = in ? prm.ws_q[o] : 0.0;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int rb = rb0 + u;
+        if (rb < prm.n_row_blocks) {
+          const int64_t r0 = static_cast<int64_t>(rb) * prm.rows_per_block;
+          const int64_t nb = (r0 + prm.rows_per_block < prm.b) ? prm.rows_per_block : prm.b - r0;
+          const double nn = static_cast<double>(n + nb);
+          const double w_mean = static_cast<double>(nb) / nn;
+          const double delta = mu[u] - mean;
+          mean += delta * w_mean;
+          m2 += mm[u] + delta * delta * (static_cast<double>(n) * w_mean);
+          q += qq[u];
+          n += nb;
+        }
+      }
     }
     const float gb = static_cast<float>(mean);
     prm.gbar[c] = gb;
     a = static_cast<double>(gb) * static_cast<double>(gb);
     s = m2;
   }
-  block_reduce3<kWarps>(a, s, q, red);
+  block_reduce3<kPsThreads / 32>(a, s, q, red);
   if (threadIdx.x == 0) {
     double* out = prm.chunk_out + static_cast<int64_t>(blockIdx.x) * 4;
     out[0] = a;
