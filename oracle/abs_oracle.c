@@ -30,6 +30,11 @@
  *                          the b_{k+1} display after Eq. 3).
  *   abs_oracle_adamw       the AdamW lines of Algorithm 1.
  *   abs_oracle_round_batch the three rounding lines of Algorithm 1's If branch.
+ *   abs_oracle_clip_scale  global-norm gradient clipping as used in the paper's experiments
+ *                          (Sec. 5 "gradient clipping"; "Gradient clipping 1.0" in the
+ *                          hyper-parameter tables of Appendix C).  The paper gives no formula;
+ *                          the reading is the convention of the PyTorch routine its stack
+ *                          calls: scale = min(1, c / (||gbar|| + 1e-6)).
  *
  * Precision: every input is widened exactly to fp64 (bf16 by a 16-bit shift) before
  * any arithmetic; all arithmetic is fp64.  Long sums are accumulated per run of
@@ -274,6 +279,37 @@ int abs_oracle_adamw(const float* w, const float* m, const float* v, const doubl
     const double mhat = mi / c1;
     const double vhat = vi / c2;
     w_out[i] = (1.0 - lr * wd) * (double)w[i] - lr * mhat / (sqrt(vhat) + eps);
+    m_out[i] = mi;
+    v_out[i] = vi;
+  }
+  return 0;
+}
+
+/*
+ * Gradient clipping by global norm (experiments only; not part of Algorithm 1):
+ *   scale = min(1, max_norm / (sqrt(n2) + 1e-6)),  n2 = ||gbar||^2
+ * The clipped gradient scale*gbar then enters the AdamW lines unchanged.
+ */
+double abs_oracle_clip_scale(double n2, double max_norm) {
+  const double coef = max_norm / (sqrt(n2) + 1e-6);
+  return coef < 1.0 ? coef : 1.0;
+}
+
+/* AdamW on the clipped gradient scale*g (scale from abs_oracle_clip_scale). */
+int abs_oracle_adamw_clipped(const float* w, const float* m, const float* v, const double* g,
+                             int64_t d, double lr, double beta1, double beta2, double eps,
+                             double wd, int64_t step, double max_norm, double n2, double* w_out,
+                             double* m_out, double* v_out) {
+  if (!w || !m || !v || !g || d < 1 || step < 1 || !w_out || !m_out || !v_out) return -1;
+  const double scale = abs_oracle_clip_scale(n2, max_norm);
+  const double c1 = 1.0 - pow(beta1, (double)step);
+  const double c2 = 1.0 - pow(beta2, (double)step);
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < d; ++i) {
+    const double gi = scale * g[i];
+    const double mi = beta1 * (double)m[i] + (1.0 - beta1) * gi;
+    const double vi = beta2 * (double)v[i] + (1.0 - beta2) * (gi * gi);
+    w_out[i] = (1.0 - lr * wd) * (double)w[i] - lr * (mi / c1) / (sqrt(vi / c2) + eps);
     m_out[i] = mi;
     v_out[i] = vi;
   }

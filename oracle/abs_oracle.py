@@ -54,6 +54,11 @@ def lib():
         L.abs_oracle_adamw.restype = cint
         L.abs_oracle_adamw.argtypes = [ptr, ptr, ptr, ptr, i64, dbl, dbl, dbl, dbl, dbl, i64,
                                        ptr, ptr, ptr]
+        L.abs_oracle_clip_scale.restype = dbl
+        L.abs_oracle_clip_scale.argtypes = [dbl, dbl]
+        L.abs_oracle_adamw_clipped.restype = cint
+        L.abs_oracle_adamw_clipped.argtypes = [ptr, ptr, ptr, ptr, i64, dbl, dbl, dbl, dbl, dbl,
+                                               i64, dbl, dbl, ptr, ptr, ptr]
         _lib = L
     return _lib
 
@@ -149,4 +154,23 @@ def adamw(w, m, v, g, lr, beta1, beta2, eps, wd, step):
                                 _p(vo))
     if rc != 0:
         raise ValueError("abs_oracle_adamw rejected its arguments")
+    return wo, mo, vo
+
+
+def clip_scale(n2, max_norm):
+    return float(lib().abs_oracle_clip_scale(float(n2), float(max_norm)))
+
+
+def adamw_clipped(w, m, v, g, lr, beta1, beta2, eps, wd, step, max_norm, n2):
+    """AdamW on the gradient clipped to global norm max_norm (n2 = ||g||^2); fp64 (w', m', v')."""
+    w, m, v = (np.ascontiguousarray(x, dtype=np.float32) for x in (w, m, v))
+    g = np.ascontiguousarray(g, dtype=np.float64)
+    d = int(w.shape[0])
+    assert m.shape[0] == d and v.shape[0] == d and g.shape[0] == d
+    wo, mo, vo = (np.empty(d, dtype=np.float64) for _ in range(3))
+    rc = lib().abs_oracle_adamw_clipped(_p(w), _p(m), _p(v), _p(g), d, float(lr), float(beta1),
+                                        float(beta2), float(eps), float(wd), int(step),
+                                        float(max_norm), float(n2), _p(wo), _p(mo), _p(vo))
+    if rc != 0:
+        raise ValueError("abs_oracle_adamw_clipped rejected its arguments")
     return wo, mo, vo

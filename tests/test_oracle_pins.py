@@ -348,6 +348,49 @@ def test_adamw_decay_multiplies_old_weight_and_eps_outside_sqrt():
     assert mo[0] == m1 and vo[0] == v1
 
 
+def test_clipped_adamw_against_torch_clip_grad_norm():
+    """torch.nn.utils.clip_grad_norm_ + torch.optim.AdamW in fp64 is the library statement of
+    clipping by global norm followed by the update."""
+    rng = np.random.default_rng(12)
+    d = 800
+    lr, b1, b2, eps, wd = [float(np.float32(x)) for x in (1e-3, 0.9, 0.95, 1e-8, 0.1)]
+    for gscale, max_norm in ((0.5, 1.0), (0.001, 1.0), (0.2, 0.25)):
+        w32 = (0.02 * rng.standard_normal(d)).astype(np.float32)
+        m32 = (0.01 * rng.standard_normal(d)).astype(np.float32)
+        v32 = (1e-4 * rng.random(d)).astype(np.float32)
+        g = gscale * rng.standard_normal(d)
+        n2 = float(np.dot(g, g))
+        p = torch.nn.Parameter(torch.from_numpy(w32.astype(np.float64)))
+        opt = torch.optim.AdamW([p], lr=lr, betas=(b1, b2), eps=eps, weight_decay=wd)
+        p.grad = torch.zeros(d, dtype=torch.float64)
+        opt.step()
+        st = opt.state[p]
+        with torch.no_grad():
+            p.copy_(torch.from_numpy(w32.astype(np.float64)))
+            st["exp_avg"].copy_(torch.from_numpy(m32.astype(np.float64)))
+            st["exp_avg_sq"].copy_(torch.from_numpy(v32.astype(np.float64)))
+            st["step"].fill_(4)
+        p.grad = torch.from_numpy(g.copy())
+        total = torch.nn.utils.clip_grad_norm_([p], max_norm)
+        assert float(total) == pytest.approx(math.sqrt(n2), rel=1e-13)
+        scale = orc.clip_scale(n2, max_norm)
+        np.testing.assert_allclose(p.grad.numpy(), scale * g, rtol=1e-13, atol=0)
+        assert (scale < 1.0) == (math.sqrt(n2) + 1e-6 > max_norm)
+        opt.step()
+        wo, mo, vo = orc.adamw_clipped(w32, m32, v32, g, lr, b1, b2, eps, wd, 5, max_norm, n2)
+        np.testing.assert_allclose(wo, p.detach().numpy(), rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(mo, st["exp_avg"].numpy(), rtol=1e-12, atol=1e-18)
+        np.testing.assert_allclose(vo, st["exp_avg_sq"].numpy(), rtol=1e-12, atol=1e-20)
+    # no clipping needed: identical to the plain update
+    g = 1e-3 * rng.standard_normal(d)
+    a = orc.adamw_clipped(w32, m32, v32, g, lr, b1, b2, eps, wd, 3, 1.0, float(np.dot(g, g)))
+    b = orc.adamw(w32, m32, v32, g, lr, b1, b2, eps, wd, 3)
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)
+    assert orc.clip_scale(4.0, 1.0) == pytest.approx(1.0 / (2.0 + 1e-6), rel=1e-15)
+    assert orc.clip_scale(0.0, 1.0) == 1.0
+
+
 # ------------------------------------------------------------------- thread independence
 def test_thread_count_does_not_change_results():
     code = (
