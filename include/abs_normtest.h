@@ -131,6 +131,23 @@ int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t
                    const abs_adamw_hparams* hparams, int64_t step, abs_stream_t stream);
 
 /*
+ * AdamW on the gradient clipped by global norm -- what the paper's experiments add to
+ * Algorithm 1 (Sec. 5 "gradient clipping"; "Gradient clipping 1.0" in the hyper-parameter
+ * tables of Appendix C).  The paper prints no formula; this follows the convention of the
+ * PyTorch routine its training stack calls:
+ *   scale = min(1, max_norm / (||gbar|| + 1e-6));   then abs_adamw_step with scale*gbar.
+ * ||gbar||^2 is read on the device from `stats_in`, the stats_out buffer that a preceding
+ * abs_norm_test on the same stream wrote for this gbar (its ABS_STAT_N2 slot), so the
+ * sequence norm test -> clipped update needs no host round trip.  Clipping needs the
+ * global norm before the first coordinate is updated, which is why it is a second pass
+ * (28 B per coordinate) and not part of the fused call.
+ *   max_norm   finite, > 0;   stats_in  device, 8-byte aligned;   rest as abs_adamw_step
+ */
+int abs_adamw_step_clipped(float* params, const float* gbar, float* m, float* v, int64_t d,
+                           const abs_adamw_hparams* hparams, int64_t step, double max_norm,
+                           const void* stats_in, abs_stream_t stream);
+
+/*
  * The fused step: abs_norm_test and abs_adamw_step in one pass, so gradients and
  * optimizer state cross HBM once.  Arguments as above; gbar_out may be NULL (the mean
  * then lives only in registers).  The diagnostic Q is not computed here: its slots in

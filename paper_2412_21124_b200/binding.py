@@ -63,6 +63,8 @@ def lib():
     L.abs_norm_test.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64, ptr, ptr, ptr, ptr]
     L.abs_adamw_step.restype = cint
     L.abs_adamw_step.argtypes = [ptr, ptr, ptr, ptr, i64, ptr, i64, ptr]
+    L.abs_adamw_step_clipped.restype = cint
+    L.abs_adamw_step_clipped.argtypes = [ptr, ptr, ptr, ptr, i64, ptr, i64, dbl, ptr, ptr]
     L.abs_normtest_adamw.restype = cint
     L.abs_normtest_adamw.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64, ptr, ptr, ptr,
                                      ptr, ptr, ptr, ptr, i64, ptr]
@@ -179,6 +181,20 @@ def abs_adamw_step(params, gbar, m, v, hparams, step, stream=None):
                               ctypes.byref(hp), int(step), _stream(stream))
     if rc != ABS_OK:
         raise AbsError(rc, "abs_adamw_step")
+
+
+def abs_adamw_step_clipped(params, gbar, m, v, hparams, step, max_norm, stats_in, stream=None):
+    """AdamW on gbar clipped to global norm max_norm; ||gbar||^2 is read on the device from
+    `stats_in` (the stats_out of the abs_norm_test that produced gbar)."""
+    d = params.numel()
+    for t, name in ((params, "params"), (gbar, "gbar"), (m, "m"), (v, "v")):
+        _check_f32_vec(t, d, name)
+    hp = _hparams(hparams)
+    rc = lib().abs_adamw_step_clipped(params.data_ptr(), gbar.data_ptr(), m.data_ptr(),
+                                      v.data_ptr(), d, ctypes.byref(hp), int(step),
+                                      float(max_norm), stats_in.data_ptr(), _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_adamw_step_clipped")
 
 
 def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v, hparams,

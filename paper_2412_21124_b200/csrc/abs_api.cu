@@ -290,8 +290,10 @@ int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dty
                        gbar_out, b_next_out, params, m, v, hparams, step, true, stream);
 }
 
-int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t d,
-                   const abs_adamw_hparams* hparams, int64_t step, abs_stream_t stream) {
+namespace {
+int run_adamw(float* params, const float* gbar, float* m, float* v, int64_t d,
+              const abs_adamw_hparams* hparams, int64_t step, const double* n2_dev,
+              double max_norm, abs_stream_t stream) {
   if (!params || !gbar || !m || !v) return ABS_ERR_NULL;
   if (d < 1) return ABS_ERR_RANGE;
   const int rc = check_hparams(hparams, step);
@@ -309,10 +311,27 @@ int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t
   if (blocks > cap) blocks = cap;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid(static_cast<unsigned>(blocks)), block(kThreads);
-  const cudaError_t e = vec ? launch_pdl(adamw_kernel<true>, grid, block, st, params, gbar, m, v, d, a)
-                            : launch_pdl(adamw_kernel<false>, grid, block, st, params, gbar, m, v, d, a);
+  const cudaError_t e =
+      vec ? launch_pdl(adamw_kernel<true>, grid, block, st, params, gbar, m, v, d, a, n2_dev, max_norm)
+          : launch_pdl(adamw_kernel<false>, grid, block, st, params, gbar, m, v, d, a, n2_dev, max_norm);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
+}
+}  // namespace
+
+int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t d,
+                   const abs_adamw_hparams* hparams, int64_t step, abs_stream_t stream) {
+  return run_adamw(params, gbar, m, v, d, hparams, step, nullptr, 0.0, stream);
+}
+
+int abs_adamw_step_clipped(float* params, const float* gbar, float* m, float* v, int64_t d,
+                           const abs_adamw_hparams* hparams, int64_t step, double max_norm,
+                           const void* stats_in, abs_stream_t stream) {
+  if (!stats_in) return ABS_ERR_NULL;
+  if (!std::isfinite(max_norm) || !(max_norm > 0.0)) return ABS_ERR_RANGE;
+  if (misaligned(stats_in, 8)) return ABS_ERR_ALIGN;
+  return run_adamw(params, gbar, m, v, d, hparams, step,
+                   static_cast<const double*>(stats_in) + ABS_STAT_N2, max_norm, stream);
 }
 
 int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs_dtype dtype,

@@ -166,6 +166,18 @@ def test_adamw_and_fused_reject_hparams(L, hp, step, status):
     assert L.abs_normtest_adamw(*args) == status
 
 
+def test_clipped_adamw_rejects(L):
+    hp = _hp()
+    r = ctypes.byref(hp)
+    f = L.abs_adamw_step_clipped
+    assert f(FAKE, FAKE, FAKE, FAKE, 10, r, 1, 1.0, None, None) == binding.ABS_ERR_NULL
+    assert f(FAKE, FAKE, FAKE, FAKE, 10, r, 1, 0.0, FAKE, None) == binding.ABS_ERR_RANGE
+    assert f(FAKE, FAKE, FAKE, FAKE, 10, r, 1, math.nan, FAKE, None) == binding.ABS_ERR_RANGE
+    assert f(FAKE, FAKE, FAKE, FAKE, 10, r, 1, 1.0, FAKE + 4, None) == binding.ABS_ERR_ALIGN
+    assert f(None, FAKE, FAKE, FAKE, 10, r, 1, 1.0, FAKE, None) == binding.ABS_ERR_NULL
+    assert f(FAKE, FAKE, FAKE, FAKE, 10, r, 0, 1.0, FAKE, None) == binding.ABS_ERR_RANGE
+
+
 def test_adamw_rejects_pointers(L):
     hp = _hp()
     r = ctypes.byref(hp)

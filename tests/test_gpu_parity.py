@@ -11,7 +11,8 @@ import torch
 import paper_2412_21124_b200 as absnt
 from oracle import abs_oracle as orc
 from paper_2412_21124_b200 import synth
-from tests.util import (assert_sum_close, assert_vec_close, margin_ok, oracle_adamw, to_host)
+from tests.util import (assert_sum_close, assert_vec_close, f32, margin_ok, oracle_adamw,
+                        to_host)
 
 pytestmark = pytest.mark.gpu
 
@@ -357,6 +358,43 @@ def test_adamw_step_sequence(d, shift):
         assert_vec_close(views[2], v_ref, "v")
     for b in bufs:
         check_guards(b, d, shift)
+
+
+@pytest.mark.parametrize("max_norm", [1.0, 0.05, 1e3])
+@pytest.mark.parametrize("d,shift", [(100_003, 0), (50_001, 1)])
+def test_norm_test_then_clipped_adamw(max_norm, d, shift):
+    """Clipping by global norm (what the paper's experiments add to Algorithm 1): the norm
+    test writes gbar and ||gbar||^2, the clipped update reads both on the device."""
+    K, eta, b_cur, step = 4, 0.1, 64, 6
+    grads, ref = make_case(K, d, torch.bfloat16, eta, b_cur, seed=1250 + d % 7)
+    p, m, v = synth.adam_state(d, 1251, DEV, zero_moments=False)
+    bufs, views = [], []
+    for t in (p, m, v):
+        b, w = guarded(d, shift=shift)
+        w.copy_(t)
+        bufs.append(b)
+        views.append(w)
+    p0, m0, v0 = (to_host(x) for x in views)
+    stats = absnt.alloc_stats(d, 1, DEV)
+    gbar = torch.empty(d, dtype=torch.float32, device=DEV)
+    b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+    absnt.abs_norm_test(grads, eta, b_cur, stats, gbar, b_next)
+    absnt.abs_adamw_step_clipped(views[0], gbar, views[1], views[2], HP, step, max_norm, stats)
+    torch.cuda.synchronize()
+    scale = orc.clip_scale(ref["n2"], max_norm)
+    assert (scale < 1.0) == (max_norm < 1e3)
+    w_ref, m_ref, v_ref = orc.adamw_clipped(p0, m0, v0, ref["gbar"], f32(HP["lr"]), f32(HP["beta1"]),
+                                            f32(HP["beta2"]), f32(HP["eps"]),
+                                            f32(HP["weight_decay"]), step, max_norm, ref["n2"])
+    assert_vec_close(views[0], w_ref, "params")
+    assert_vec_close(views[1], m_ref, "m")
+    assert_vec_close(views[2], v_ref, "v")
+    for b in bufs:
+        check_guards(b, d, shift)
+    if max_norm == 1e3:  # inactive clipping is the plain update, bit for bit
+        q, mq, vq = (torch.from_numpy(x).to(DEV) for x in (p0, m0, v0))
+        absnt.abs_adamw_step(q, gbar, mq, vq, HP, step)
+        assert torch.equal(q, views[0]) and torch.equal(mq, views[1]) and torch.equal(vq, views[2])
 
 
 # --------------------------------------------------------------------- per-sample form
