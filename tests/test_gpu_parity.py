@@ -562,3 +562,49 @@ def test_config3_full_size_fsdp_shards():
             if eta == 0.1:
                 assert dev_b_next == ob
     assert decided >= 2
+
+
+def test_more_than_2_to_31_coordinates():
+    """64-bit indexing: d just above 2^31 with shard boundaries on both sides of 2^31.  The
+    unfused test is checked shard by shard against the oracle; the fused call must reproduce the
+    sums and is checked element-wise on three 1M-coordinate windows (start, across 2^31, end)."""
+    d = (1 << 31) + 3 * 4096 + 5
+    K, eta, b_cur, step = 2, 0.1, 64, 3
+    offs = [0, (1 << 30) + 17, (1 << 31) - 1000, d]
+    grads = synth.worker_grads([d], K, torch.bfloat16, 4000, DEV)
+    stats = absnt.alloc_stats(d, 3, DEV)
+    gbar = torch.empty(d, dtype=torch.float32, device=DEV)
+    b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+    absnt.abs_norm_test(grads, eta, b_cur, stats, gbar, b_next, shard_offsets=offs)
+    torch.cuda.synchronize()
+    got = absnt.read_stats(stats, 3)
+    tot = [0.0, 0.0]
+    for s in range(3):
+        lo, hi = offs[s], offs[s + 1]
+        ref = orc.norm_test([to_host(g[lo:hi]) for g in grads], eta, b_cur, want_gbar=False)
+        for j, key in enumerate(("n2", "S")):
+            assert abs(got["shards"][s][j] - ref[key]) <= 1e-6 * ref[key], (s, key)
+            tot[j] += ref[key]
+    assert_sum_close(got["n2"], tot[0], "n2")
+    assert_sum_close(got["S"], tot[1], "S")
+    ob, oT, _ = orc.decide(tot[1], tot[0], K, eta, b_cur)
+    if margin_ok(oT, b_cur):
+        assert int(b_next.item()) == ob
+
+    p, m, v = synth.adam_state(d, 4001, DEV, zero_moments=False)
+    windows = [(0, 1 << 20), ((1 << 31) - (1 << 19), (1 << 31) + (1 << 19)), (d - (1 << 20), d)]
+    before = [[to_host(x[lo:hi]) for x in (p, m, v)] for lo, hi in windows]
+    stats2 = absnt.alloc_stats(d, 1, DEV)
+    gbar.fill_(-1.0)
+    absnt.abs_normtest_adamw(grads, eta, b_cur, stats2, gbar, b_next, p, m, v, HP, step)
+    torch.cuda.synchronize()
+    got2 = absnt.read_stats(stats2)
+    assert_sum_close(got2["n2"], tot[0], "n2 fused")
+    assert_sum_close(got2["S"], tot[1], "S fused")
+    for (lo, hi), (p0, m0, v0) in zip(windows, before):
+        ref = orc.norm_test([to_host(g[lo:hi]) for g in grads], eta, b_cur)
+        assert_vec_close(gbar[lo:hi], ref["gbar"], "gbar window")
+        w_ref, m_ref, v_ref = oracle_adamw(orc, p0, m0, v0, ref["gbar"], HP, step)
+        assert_vec_close(p[lo:hi], w_ref, "params window")
+        assert_vec_close(m[lo:hi], m_ref, "m window")
+        assert_vec_close(v[lo:hi], v_ref, "v window")
