@@ -140,13 +140,14 @@ cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
   // predicated K buckets (K=12: 5.46 vs 5.80 TB/s), and the unfused test -- 20 B per
   // coordinate at K=8 bf16, i.e. twice the coordinates per second -- is bound by instruction
   // issue, where the per-tile bookkeeping of the staged kernel costs 10% (5.95 vs 6.60 TB/s).
-  constexpr int tile =
-      (!ADAM || (bulk_tile<GT, KB, ADAM>() == 512 && !EXACT)) ? 0 : bulk_tile<GT, KB, ADAM>();
+  constexpr BulkShape shape = bulk_shape<GT, KB, ADAM>();
+  constexpr int tile = (!ADAM || (shape.tile == 512 && !EXACT)) ? 0 : shape.tile;
   if constexpr (tile > 0) {
     constexpr size_t smem =
-        static_cast<size_t>(kBulkStages) * bulk_stage_bytes<GT, KB, ADAM>(tile);
-    return launch_pdl_smem(normtest_bulk_kernel<GT, KB, EXACT, ADAM, !ADAM, tile>, grid,
-                           dim3(tile / 4), smem, st, prm);
+        static_cast<size_t>(shape.stages) * bulk_stage_bytes<GT, KB, ADAM>(tile);
+    return launch_pdl_smem(
+        normtest_bulk_kernel<GT, KB, EXACT, ADAM, !ADAM, tile, shape.stages, shape.ctas>, grid,
+        dim3(tile / 4), smem, st, prm);
   } else {
     return launch_pdl(normtest_stream_kernel<GT, KB, EXACT, ADAM, !ADAM>, grid, dim3(kThreads), st,
                       prm);

@@ -24,7 +24,6 @@
 
 namespace absnt {
 
-constexpr int kBulkStages = 3;
 constexpr int kBulkWaitLimit = 1 << 22;  // mbarrier polls before giving up
 constexpr int kSmemPerSM = 224 * 1024;   // budget for dynamic shared memory per SM
 
@@ -33,15 +32,18 @@ template <typename GT, int KB, bool ADAM>
 __host__ __device__ constexpr int bulk_stage_bytes(int tile) {
   return tile * (KB * static_cast<int>(sizeof(typename GT::scalar)) + (ADAM ? 12 : 0) + 4);
 }
-// Tile size (coordinates per stage, 4 per thread): 1024 with two 256-thread CTAs per SM
-// where three stages of both fit; else 512 with three 128-thread CTAs per SM; else 0 (the
-// register-direct kernel is used).  With a single resident CTA the staging loses to the
-// register-direct kernel, so those shapes are not offered.
+// Shape of the staged kernel for one (dtype, K, fused) combination: coordinates per stage
+// (4 per thread), stages per CTA, CTAs per SM.  tile == 0: not offered.  Measured and
+// rejected: a single resident CTA with three stages (bf16 K=16: 5.83 vs 6.63 TB/s of the
+// register-direct kernel) and two CTAs with two stages (bf16 K=32: 5.85 vs 6.31 TB/s).
+struct BulkShape {
+  int tile, stages, ctas;
+};
 template <typename GT, int KB, bool ADAM>
-__host__ __device__ constexpr int bulk_tile() {
-  return 2 * kBulkStages * bulk_stage_bytes<GT, KB, ADAM>(1024) <= kSmemPerSM
-             ? 1024
-             : (3 * kBulkStages * bulk_stage_bytes<GT, KB, ADAM>(512) <= kSmemPerSM ? 512 : 0);
+__host__ __device__ constexpr BulkShape bulk_shape() {
+  if (2 * 3 * bulk_stage_bytes<GT, KB, ADAM>(1024) <= kSmemPerSM) return {1024, 3, 2};
+  if (3 * 3 * bulk_stage_bytes<GT, KB, ADAM>(512) <= kSmemPerSM) return {512, 3, 3};
+  return {0, 0, 0};
 }
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {
@@ -124,10 +126,11 @@ struct BulkGrad<F32> {
   }
 };
 
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ, int TILE>
-__global__ void __launch_bounds__(TILE / 4, (TILE == 1024 ? 2 : 3))
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ, int TILE, int STAGES, int CTAS>
+__global__ void __launch_bounds__(TILE / 4, CTAS)
     normtest_bulk_kernel(const __grid_constant__ StreamParams prm) {
   constexpr int kBulkTile = TILE;
+  constexpr int kBulkStages = STAGES;
   constexpr int NT = TILE / 4;  // threads
   constexpr int GB = kBulkTile * static_cast<int>(sizeof(typename GT::scalar));  // gradient segment
   constexpr int FB = kBulkTile * 4;                                              // fp32 segment
