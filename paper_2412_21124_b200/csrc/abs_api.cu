@@ -5,6 +5,7 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 #include <utility>
 
 #include "abs_device.cuh"
@@ -166,7 +167,10 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
     case 4: return launch_one<GT, 4, true, ADAM>(prm, st);
     case 8: return launch_one<GT, 8, true, ADAM>(prm, st);
     case 16: return launch_one<GT, 16, true, ADAM>(prm, st);
-    case 32: return launch_one<GT, 32, true, ADAM>(prm, st);
+    case 32:
+      // bf16, K=32: four coordinates per thread-row (see BF16H)
+      if constexpr (std::is_same<GT, BF16>::value) return launch_one<BF16H, 32, true, ADAM>(prm, st);
+      else return launch_one<GT, 32, true, ADAM>(prm, st);
     default:
       if (K < 8) return launch_one<GT, 8, false, ADAM>(prm, st);
       if (K < 16) return launch_one<GT, 16, false, ADAM>(prm, st);

@@ -137,6 +137,8 @@ __device__ __forceinline__ float mean_of_sum(float s, float inv_K, float neg_K) 
 struct F32 {
   static constexpr int kVec = 4; // elements per 16 bytes
   using scalar = float;
+  using raw_t = uint4;
+  static __device__ __forceinline__ raw_t load_vec(const void* p) { return ld_once_16(p); }
   using sum_t = double; // fp32 addends: only an fp64 sum keeps the mean correctly rounded
   template <bool POW2>
   static __device__ __forceinline__ float mean(double s, const StreamParams& prm) {
@@ -152,6 +154,8 @@ struct F32 {
 struct BF16 {
   static constexpr int kVec = 8;
   using scalar = uint16_t;
+  using raw_t = uint4;
+  static __device__ __forceinline__ raw_t load_vec(const void* p) { return ld_once_16(p); }
   using sum_t = float; // 8-bit significands: fp32 partial sums are exact within 13 binades
   template <bool POW2>
   static __device__ __forceinline__ float mean(float s, const StreamParams& prm) {
@@ -164,6 +168,30 @@ struct BF16 {
   static __device__ __forceinline__ float load1(const void* base, int64_t i) {
     return __uint_as_float(
         static_cast<uint32_t>(__ldg(reinterpret_cast<const uint16_t*>(base) + i)) << 16);
+  }
+};
+// bf16 gradients taken four coordinates (8 bytes) per thread-row instead of eight: half the
+// registers per worker, so that the K=32 kernels keep two CTAs per SM resident.
+struct BF16H {
+  static constexpr int kVec = 4;
+  using scalar = uint16_t;
+  using raw_t = uint2;
+  using sum_t = float;
+  static __device__ __forceinline__ raw_t load_vec(const void* p) {
+    uint2 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
+    return r;
+  }
+  template <bool POW2>
+  static __device__ __forceinline__ float mean(float s, const StreamParams& prm) {
+    return mean_of_sum<POW2>(s, prm.inv_Kf, prm.neg_Kf);
+  }
+  static __device__ __forceinline__ float elem(const uint2& r, int e) {
+    const uint32_t w = (e >> 1) ? r.y : r.x;
+    return (e & 1) ? bf16_hi(w) : bf16_lo(w);
+  }
+  static __device__ __forceinline__ float load1(const void* base, int64_t i) {
+    return BF16::load1(base, i);
   }
 };
 

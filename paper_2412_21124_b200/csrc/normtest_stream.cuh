@@ -137,11 +137,11 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
     float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
 
     if (cg.aligned && (row_lo + NT * V <= hi)) {
-      uint4 raw[KB];
+      typename GT::raw_t raw[KB];
 #pragma unroll
       for (int k = 0; k < KB; ++k)
         if (EXACT || k < K)
-          raw[k] = ld_once_16(reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) + base);
+          raw[k] = GT::load_vec(reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) + base);
       float4 pw[NF4], pm[NF4], pv[NF4];
       if (ADAM) {
         if (V == 8 && wide) {
@@ -232,7 +232,7 @@ __device__ __forceinline__ void write_chunk_record(const StreamParams& prm, int 
 }
 
 template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
-__global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : (KB <= 16 ? 2 : 1)))
+__global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : ((KB <= 16 || GT::kVec * sizeof(typename GT::scalar) <= 8) ? 2 : 1)))
     normtest_stream_kernel(const __grid_constant__ StreamParams prm) {
   __shared__ double red[kWarps * 3];
   const int K = EXACT ? KB : prm.K;
