@@ -179,8 +179,8 @@ int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dty
  * Arguments, results and status codes are those of abs_normtest_adamw, except:
  *   stats_out   device, only (ABS_STATS_HEADER + n_shards*ABS_SHARD_STRIDE) doubles
  *               (header and shard records; no scratch tail), 16-byte aligned
- *   limit       ceil(d/c) + n_shards must not exceed ABS_NOALLOC_MAX_CHUNKS, where c = 16384
- *               for d >= 2^23 and 4096 below (any d up to about 2.1e9); larger problems
+ *   limit       ceil(d/c) + n_shards must not exceed ABS_NOALLOC_MAX_CHUNKS, where c = 8192
+ *               for d >= 2^23 and 4096 below (any d up to about 1.07e9); larger problems
  *               return ABS_ERR_TOO_LARGE and launch nothing
  * Results are bit-identical to abs_normtest_adamw on the same inputs.
  *

@@ -24,9 +24,15 @@ int cuda_fail(cudaError_t e) {
   return ABS_ERR_CUDA;
 }
 
-// Elements per reduction chunk.  A function of d alone, so that the summation tree --
-// and with it every output bit -- depends only on the problem, not on the launch.
-int chunk_elems_for(int64_t d) { return d >= (int64_t{1} << 23) ? 16384 : 4096; }
+// Elements per reduction chunk (= the work of one CTA).  A function of the problem (d and
+// the entry point) alone, so that the summation tree -- and with it every output bit --
+// never depends on the launch.  Measured at d=124M: the fused kernels like 8192 (+0.5..2%
+// over 16384; 4096 costs the staged kernel 4% in pipeline fill and drain); the unfused
+// test, bound by instruction issue, likes 16384 (the per-chunk reduction costs it 2.5% at
+// 8192).  abs_stats_bytes sizes the scratch for the smaller of the two.
+int chunk_elems_for(int64_t d, bool fused) {
+  return d >= (int64_t{1} << 23) ? (fused ? 8192 : 16384) : 4096;
+}
 
 bool finite_nonneg(float x) { return std::isfinite(x) && x >= 0.f; }
 
@@ -86,11 +92,11 @@ struct Layout {
 };
 
 // Validates the shard table and cuts the shards into chunks.
-int make_layout(int64_t d, const int64_t* shard_offsets, int n_shards, Layout* L) {
+int make_layout(int64_t d, const int64_t* shard_offsets, int n_shards, bool fused, Layout* L) {
   if (!shard_offsets) n_shards = 1;
   if (n_shards < 1 || n_shards > ABS_MAX_SHARDS) return ABS_ERR_RANGE;
   L->n_shards = n_shards;
-  L->chunk_elems = chunk_elems_for(d);
+  L->chunk_elems = chunk_elems_for(d, fused);
   if (!shard_offsets) {
     L->shard_off[0] = 0;
     L->shard_off[1] = d;
@@ -204,7 +210,7 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
     return ABS_ERR_ALIGN;
 
   Layout L;
-  const int rc = make_layout(d, shard_offsets, n_shards, &L);
+  const int rc = make_layout(d, shard_offsets, n_shards, fused, &L);
   if (rc != ABS_OK) return rc;
 
   double* stats = static_cast<double*>(stats_out);
@@ -263,7 +269,7 @@ extern "C" {
 
 size_t abs_stats_bytes(int64_t d, int n_shards) {
   if (d < 1 || n_shards < 1 || n_shards > ABS_MAX_SHARDS) return 0;
-  const int ce = chunk_elems_for(d);
+  const int ce = chunk_elems_for(d, true);
   const int64_t max_chunks = (d + ce - 1) / ce + n_shards;
   return sizeof(double) * (ABS_STATS_HEADER + static_cast<size_t>(n_shards) * ABS_SHARD_STRIDE +
                            static_cast<size_t>(max_chunks) * 4);
@@ -506,7 +512,7 @@ extern "C" int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64
   if (misaligned(params, 4) || misaligned(m, 4) || misaligned(v, 4)) return ABS_ERR_ALIGN;
 
   Layout L;
-  rc = make_layout(d, shard_offsets, n_shards, &L);
+  rc = make_layout(d, shard_offsets, n_shards, true, &L);
   if (rc != ABS_OK) return rc;
   if (L.n_chunks > ABS_NOALLOC_MAX_CHUNKS) return ABS_ERR_TOO_LARGE;
 

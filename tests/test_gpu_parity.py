@@ -204,7 +204,9 @@ def test_large_d_uses_bigger_chunks():
     # d >= 2^23 switches the reduction chunk; several chunks plus a ragged tail
     got, _ = run_and_check(2, (1 << 23) + 12_345, torch.bfloat16, fused=True, seed=650,
                            zero_moments=False, step=9)
-    assert got["n_chunks"] == 513
+    assert got["n_chunks"] == 1026  # 8192 per chunk in the fused call
+    got, _ = run_and_check(2, (1 << 23) + 12_345, torch.bfloat16, fused=False, seed=651)
+    assert got["n_chunks"] == 513   # 16384 per chunk in the unfused test
 
 
 # ----------------------------------------------------------------------------- shards

@@ -64,7 +64,7 @@ def _run_pair(K, d, dtype, n_shards, step, seed):
 def test_noalloc_matches_existing_entry_point_twice_in_a_row():
     assert torch.cuda.is_available(), "GPU tests need a CUDA device"
     torch.cuda.set_device(0)
-    # first call: large problem (16384-element chunks), several shards
+    # first call: large problem (8192-element chunks), several shards
     _run_pair(K=8, d=(1 << 23) + 40_001, dtype=torch.bfloat16, n_shards=4, step=7, seed=41)
     # second call straight after it: smaller problem, other dtype and chunk size; the shared
     # array still holds the first call's records beyond this call's chunks
@@ -77,7 +77,7 @@ def test_noalloc_rejects_problems_beyond_the_builtin_array():
     fake = 0x10000  # never dereferenced: the size check comes before any launch
     table = (ctypes.c_void_p * 2)(fake, fake)
     hp = binding.abs_adamw_hparams(1e-3, 0.9, 0.999, 1e-8, 0.1)
-    too_many = (binding.ABS_NOALLOC_MAX_CHUNKS + 1) * 16384
+    too_many = (binding.ABS_NOALLOC_MAX_CHUNKS + 1) * 8192
     rc = L.abs_normtest_adamw_noalloc(table, 2, too_many, binding.ABS_BF16, None, 1, 0.1, 8,
                                       fake, None, fake, fake, fake, fake, ctypes.byref(hp), 1,
                                       None)
