@@ -161,6 +161,15 @@ cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
   }
 }
 
+// More than 16 workers: the split kernel, four coordinates per thread-row (bf16 gradients
+// are then read with 8-byte loads).
+template <typename GT, bool EXACT, bool ADAM>
+cudaError_t launch_split(const StreamParams& prm, cudaStream_t st) {
+  using G4 = typename std::conditional<std::is_same<GT, BF16>::value, BF16H, GT>::type;
+  return launch_pdl(normtest_split_kernel<G4, 32, EXACT, ADAM, !ADAM>,
+                    dim3(static_cast<unsigned>(prm.n_chunks)), dim3(kThreads), st, prm);
+}
+
 // The fused kernel leaves Q out (its stats slot reads NaN): at the power cap the K extra
 // multiply-adds per coordinate cost about 1% of bandwidth.  The unfused test computes it.
 template <typename GT, bool ADAM>
@@ -173,14 +182,15 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
     case 4: return launch_one<GT, 4, true, ADAM>(prm, st);
     case 8: return launch_one<GT, 8, true, ADAM>(prm, st);
     case 16: return launch_one<GT, 16, true, ADAM>(prm, st);
-    case 32:
-      // bf16, K=32: four coordinates per thread-row (see BF16H)
-      if constexpr (std::is_same<GT, BF16>::value) return launch_one<BF16H, 32, true, ADAM>(prm, st);
-      else return launch_one<GT, 32, true, ADAM>(prm, st);
+    case 32: return launch_split<GT, true, ADAM>(prm, st);
     default:
       if (K < 8) return launch_one<GT, 8, false, ADAM>(prm, st);
       if (K < 16) return launch_one<GT, 16, false, ADAM>(prm, st);
-      return launch_one<GT, 32, false, ADAM>(prm, st);
+      // 17..31 workers.  Measured at K=20/24: the run-time loop over groups of 8 wins for
+      // fp32 gradients (5.27 vs 4.41 TB/s) and loses for bf16, whose 8-byte loads leave too
+      // few bytes in flight (4.20 vs 4.73 TB/s).
+      if constexpr (std::is_same<GT, F32>::value) return launch_split<GT, false, ADAM>(prm, st);
+      else return launch_one<GT, 32, false, ADAM>(prm, st);
   }
 }
 

@@ -44,11 +44,38 @@ __device__ __forceinline__ float coord_math(const float (&g)[KB], int K, const S
   return mean;
 }
 
+// The same three quantities with the shifted one-pass form used for many workers:
+//   c = g_0;  S_i = sum_k (g_k - c)^2 - K (gbar - c)^2
+// so that the K values need not all be live at once.  The cancellation is bounded: the
+// first sum exceeds S_i by at most a factor of about K (when g_0 itself is the outlier).
+// K identical values give exactly zero.  The operation order is that of the vector path of
+// chunk_rows_split, so both give identical bits.
+template <typename GT, int KB, bool EXACT, bool WITHQ>
+__device__ __forceinline__ float coord_math_split(const float (&g)[KB], int K,
+                                                  const StreamParams& prm, float& dev2, float& sq) {
+  typename GT::sum_t s = 0;
+  const float c = g[0];
+  float s2 = 0.f;
+  sq = 0.f;
+#pragma unroll
+  for (int k = 0; k < KB; ++k)
+    if (EXACT || k < K) {
+      s += static_cast<typename GT::sum_t>(g[k]);
+      const float dv = g[k] - c;
+      s2 = fmaf(dv, dv, s2);
+      if (WITHQ) sq = fmaf(g[k], g[k], sq);
+    }
+  const float mean = GT::template mean<false>(s, prm);
+  const float dm = mean - c;
+  dev2 = fmaxf(fmaf(prm.neg_Kf * dm, dm, s2), 0.f);
+  return mean;
+}
+
 // The V coordinates of one thread-row with element-wise, bounds-checked accesses: used for
 // rows that are ragged (end of a shard) or whose streams are not 16-byte aligned.  Same
 // arithmetic in the same order as the vector path, so both give identical bits.  Kept out
 // of line so that its registers do not weigh on the vector path.
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ, bool SPLIT = false>
 __device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t base, int64_t hi,
                                         float* sums /* n2, S, Q of this thread-row */) {
   constexpr int V = GT::kVec;
@@ -60,7 +87,8 @@ __device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t 
 #pragma unroll
     for (int k = 0; k < KB; ++k) g[k] = (EXACT || k < K) ? GT::load1(prm.grads[k], i) : 0.f;
     float dev2, sq;
-    const float mean = coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
+    const float mean = SPLIT ? coord_math_split<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq)
+                             : coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
     row_n2 = fmaf(mean, mean, row_n2);
     row_S += dev2;
     row_Q += sq;
@@ -245,6 +273,116 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : ((KB <= 16
     }
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
     chunk_rows_direct<GT, KB, EXACT, ADAM, WITHQ>(prm, K, cg, acc_n2, acc_S, acc_Q);
+    write_chunk_record<WITHQ>(prm, chunk, acc_n2, acc_S, acc_Q, red);
+  }
+}
+
+// Register-direct processing for many workers, or for a worker count without an unrolled
+// kernel of its own: the workers are taken in groups (two halves of 16 for K = 32; a
+// run-time loop over groups of 8 otherwise) with the shifted one-pass form of
+// coord_math_split, so only one group of gradient vectors is live per thread (two or three
+// CTAs per SM instead of one at 255 registers, and no instructions for absent workers
+// beyond the last group).
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+__device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
+                                                 const ChunkGeometry& cg, double& acc_n2,
+                                                 double& acc_S, double& acc_Q) {
+  constexpr int V = GT::kVec;
+  static_assert(V == 4, "split path: four coordinates per thread-row");
+  // exact K: compile-time halves of 16; any other K: a run-time loop over groups of 8
+  constexpr int H = EXACT ? 16 : 8;
+  static_assert(KB % H == 0, "groups");
+  const int n_groups = EXACT ? KB / H : (K + H - 1) / H;
+  const int tid = threadIdx.x;
+  const int64_t hi = cg.hi;
+
+  for (int64_t row_lo = cg.lo; row_lo < hi; row_lo += kThreads * V) {
+    const int64_t base = row_lo + static_cast<int64_t>(tid) * V;
+    float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
+    if (cg.aligned && (row_lo + kThreads * V <= hi)) {
+      typename GT::sum_t s[V];
+      float c[V], s2[V], q[V];
+#pragma unroll
+      for (int e = 0; e < V; ++e) {
+        s[e] = 0;
+        c[e] = s2[e] = q[e] = 0.f;
+      }
+      float4 pw, pm, pv;
+      if (ADAM) {  // in flight while the gradients are consumed
+        pw = ld_state_16(prm.p + base);
+        pm = ld_state_16(prm.m + base);
+        pv = ld_state_16(prm.v + base);
+      }
+#pragma unroll(EXACT ? KB / H : 1)
+      for (int h = 0; h < n_groups; ++h) {
+        typename GT::raw_t raw[H];
+#pragma unroll
+        for (int k = 0; k < H; ++k)
+          if (EXACT || h * H + k < K)
+            raw[k] = GT::load_vec(
+                reinterpret_cast<const typename GT::scalar*>(prm.grads[h * H + k]) + base);
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+#pragma unroll
+          for (int k = 0; k < H; ++k)
+            if (EXACT || h * H + k < K) {
+              const float g = GT::elem(raw[k], e);
+              if (h == 0 && k == 0) c[e] = g;
+              s[e] += static_cast<typename GT::sum_t>(g);
+              const float dv = g - c[e];
+              s2[e] = fmaf(dv, dv, s2[e]);
+              if (WITHQ) q[e] = fmaf(g, g, q[e]);
+            }
+        }
+      }
+      float gb[V];
+      float* w4 = reinterpret_cast<float*>(&pw);
+      float* m4 = reinterpret_cast<float*>(&pm);
+      float* v4 = reinterpret_cast<float*>(&pv);
+#pragma unroll
+      for (int e = 0; e < V; ++e) {
+        const float mean = GT::template mean<false>(s[e], prm);
+        const float dm = mean - c[e];
+        const float dev2 = fmaxf(fmaf(prm.neg_Kf * dm, dm, s2[e]), 0.f);
+        gb[e] = mean;
+        row_n2 = fmaf(mean, mean, row_n2);
+        row_S += dev2;
+        row_Q += q[e];
+        if (ADAM) adamw_elem(prm.adam, mean, w4[e], m4[e], v4[e]);
+      }
+      if (prm.gbar) st_stream_16(prm.gbar + base, make_float4(gb[0], gb[1], gb[2], gb[3]));
+      if (ADAM) {
+        st_stream_16(prm.p + base, pw);
+        st_stream_16(prm.m + base, pm);
+        st_stream_16(prm.v + base, pv);
+      }
+    } else if (base < hi) {
+      float sums[3];
+      scalar_row<GT, KB, EXACT, ADAM, WITHQ, true>(prm, K, base, hi, sums);
+      row_n2 = sums[0];
+      row_S = sums[1];
+      row_Q = sums[2];
+    }
+    acc_n2 += static_cast<double>(row_n2);
+    acc_S += static_cast<double>(row_S);
+    if (WITHQ) acc_Q += static_cast<double>(row_Q);
+  }
+}
+
+template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+__global__ void __launch_bounds__(kThreads, 2)
+    normtest_split_kernel(const __grid_constant__ StreamParams prm) {
+  __shared__ double red[kWarps * 3];
+  const int K = EXACT ? KB : prm.K;
+  bool waited = false;
+  for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
+    const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, K, chunk);
+    if (!waited) {
+      grid_dependency_wait();
+      waited = true;
+    }
+    double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
+    chunk_rows_split<GT, KB, EXACT, ADAM, WITHQ>(prm, K, cg, acc_n2, acc_S, acc_Q);
     write_chunk_record<WITHQ>(prm, chunk, acc_n2, acc_S, acc_Q, red);
   }
 }
