@@ -196,6 +196,15 @@ def test_misaligned_buffers(dtype, grad_shift, state_shift):
                   state_shift=state_shift)
 
 
+@pytest.mark.parametrize("K,dtype", [(32, torch.bfloat16), (32, torch.float32), (20, torch.float32)],
+                         ids=["K32-bf16", "K32-f32", "K20-f32"])
+def test_many_workers_ragged_and_misaligned(K, dtype):
+    # the split kernels: vector rows, a ragged tail, and the element-wise path of shifted buffers
+    run_and_check(K, 9_999, dtype, fused=True, seed=540 + K)
+    run_and_check(K, 9_999, dtype, fused=True, seed=541 + K, grad_shift=1, state_shift=3)
+    run_and_check(K, 9_999, dtype, fused=False, seed=542 + K, shard_offsets=[0, 5, 4101, 9_999])
+
+
 def test_fused_without_gbar_output():
     run_and_check(8, 40_000, torch.bfloat16, fused=True, seed=600, want_gbar=False)
 
