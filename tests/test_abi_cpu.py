@@ -37,6 +37,30 @@ def test_every_declared_symbol_is_exported(L):
         assert hasattr(L, n), "header declares %s but the library does not export it" % n
 
 
+def test_header_is_plain_c_and_links_from_c(L, tmp_path):
+    """The boundary is a C ABI: the header compiles as C99 and a C program can call the
+    host-side helpers of the shared library."""
+    import subprocess
+    src = tmp_path / "use_abi.c"
+    src.write_text(
+        '#include "abs_normtest.h"\n#include <stdio.h>\n'
+        "int main(void) {\n"
+        "  double T; int flags;\n"
+        "  long long b = (long long)abs_decide(4.0, 8.0, 2.0, 0.25, 3, &T, &flags);\n"
+        "  abs_adamw_hparams hp = {1e-3f, 0.9f, 0.999f, 1e-8f, 0.1f};\n"
+        "  int rc = abs_adamw_step(0, 0, 0, 0, 10, &hp, 1, 0);\n"
+        '  printf("%lld %.1f %d %lld %d %zu\\n", b, T, flags, (long long)abs_round_batch(259, 4, 16), rc,\n'
+        "         abs_stats_bytes(1, 1));\n"
+        "  return 0;\n}\n")
+    exe = tmp_path / "use_abi"
+    lib_dir = os.path.dirname(binding._build.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-I",
+                           os.path.join(ROOT, "include"), str(src), "-o", str(exe), "-L", lib_dir,
+                           "-labs_normtest", "-Wl,-rpath," + lib_dir])
+    out = subprocess.check_output([str(exe)]).decode().split()
+    assert out == ["4", "4.0", "4", "320", str(binding.ABS_ERR_NULL), str(8 * 8 + 4 * 8 + 2 * 32)]
+
+
 def test_status_strings(L):
     seen = set()
     for s in range(0, -7, -1):
