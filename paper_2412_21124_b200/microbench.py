@@ -4,7 +4,8 @@
   python -m paper_2412_21124_b200.microbench --sweep            # the d x K x dtype grid
 
 Timing: CUDA events on the launching stream around `steps` back-to-back calls after
-`warmup` calls.  Points whose working set is smaller than twice the L2 rotate over several
+`warmup` calls; calls shorter than ~50 us are captured in a CUDA graph and the replays are
+timed, so that the figure is device time and not the host's per-call cost.  Points whose working set is smaller than twice the L2 rotate over several
 independent buffer sets so that every call reads cold data.  GB/s counts algorithmic bytes:
 fused (K*s + 24) per coordinate (+4 with --gbar), normtest K*s + 4, adamw 28, persample 4
 per matrix element.
@@ -41,7 +42,8 @@ def bytes_per_call(call, d, K, esz, gbar, b):
     return 4 * b * d
 
 
-def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b=4096, dev="cuda"):
+def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b=4096, dev="cuda",
+              graph=None):
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     esz = 2 if dtype == "bf16" else 4
     nbytes = bytes_per_call(call, d, K, esz, gbar, b)
@@ -86,25 +88,49 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
     for i in range(warmup):
         one(i)
     torch.cuda.synchronize()
+    est_ms = None
     if steps is None:
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         one(0)
         e1.record()
         torch.cuda.synchronize()
-        est = max(e0.elapsed_time(e1), 1e-3)
-        steps = int(max(10, min(400, 300.0 / est)))
+        est_ms = max(e0.elapsed_time(e1), 1e-3)
+        steps = int(max(10, min(400, 300.0 / est_ms)))
+    if graph is None:  # calls shorter than ~50 us are bound by the host's per-call cost
+        graph = est_ms is not None and est_ms < 0.05
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    stream = torch.cuda.current_stream()
-    e0.record(stream)
-    for i in range(steps):
-        one(warmup + i)
-    e1.record(stream)
-    torch.cuda.synchronize()
+    if graph:
+        # capture the calls once, replay them: device-side time of back-to-back calls
+        per_graph = max(n_sets, min(steps, 64))
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(per_graph):
+                    one(i)
+        torch.cuda.current_stream().wait_stream(side)
+        replays = max(1, steps // per_graph)
+        g.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(replays):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        steps = replays * per_graph
+    else:
+        stream = torch.cuda.current_stream()
+        e0.record(stream)
+        for i in range(steps):
+            one(warmup + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     out = {"call": call, "d": d, "K": K, "dtype": dtype, "n_shards": n_shards, "gbar": bool(gbar),
-           "steps": steps, "buffer_sets": n_sets, "ms": ms, "bytes": nbytes,
-           "GBps": nbytes / (ms * 1e-3) / 1e9}
+           "steps": steps, "buffer_sets": n_sets, "cuda_graph": bool(graph), "ms": ms,
+           "bytes": nbytes, "GBps": nbytes / (ms * 1e-3) / 1e9}
     if call == "persample":
         out["b"] = b
     return out
@@ -122,13 +148,16 @@ def main(argv=None):
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--gbar", action="store_true", help="fused: also write gbar")
     ap.add_argument("--sweep", action="store_true", help="fused call over the d x K x dtype grid")
+    ap.add_argument("--graph", choices=["auto", "on", "off"], default="auto",
+                    help="time replays of a captured CUDA graph (auto: for calls under 50 us)")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device (there is no CPU fallback)")
     B.lib()
+    graph = {"auto": None, "on": True, "off": False}[args.graph]
     if not args.sweep:
         print(json.dumps(run_point(args.call, args.d, args.K, args.dtype, args.shards, args.steps,
-                                   args.warmup, args.gbar, args.b)), flush=True)
+                                   args.warmup, args.gbar, args.b, graph=graph)), flush=True)
         return
     for dtype in ("bf16", "f32"):
         esz = 2 if dtype == "bf16" else 4
@@ -138,7 +167,7 @@ def main(argv=None):
                     print(json.dumps({"call": "fused", "d": d, "K": K, "dtype": dtype,
                                       "skipped": "K*d*s + 16*d exceeds 160 GB"}), flush=True)
                     continue
-                r = run_point("fused", d, K, dtype, steps=args.steps, warmup=args.warmup)
+                r = run_point("fused", d, K, dtype, steps=args.steps, warmup=args.warmup, graph=graph)
                 print(json.dumps(r), flush=True)
                 torch.cuda.empty_cache()
 

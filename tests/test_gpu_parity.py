@@ -276,6 +276,43 @@ def test_prepared_fused_step_matches_plain_call():
         assert torch.equal(a, b)
 
 
+def test_calls_can_be_captured_in_a_cuda_graph():
+    """The library only enqueues kernels on the caller's stream, so a sequence of calls can be
+    captured once and replayed (how a launch-bound small-d loop avoids per-call host cost)."""
+    K, d = 4, 200_003
+    grads, ref = make_case(K, d, torch.bfloat16, 0.1, 64, seed=770)
+    p, m, v = synth.adam_state(d, 771, DEV, zero_moments=False)
+    p0, m0, v0 = p.clone(), m.clone(), v.clone()
+    stats = absnt.alloc_stats(d, 1, DEV)
+    gbar = torch.empty(d, dtype=torch.float32, device=DEV)
+    b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+    # eager reference (also the first, un-captured call of every kernel involved)
+    absnt.abs_normtest_adamw(grads, 0.1, 64, stats, gbar, b_next, p, m, v, HP, 4)
+    absnt.abs_adamw_step(p, gbar, m, v, HP, 5)
+    torch.cuda.synchronize()
+    want = (stats[:2].clone(), gbar.clone(), p.clone(), m.clone(), v.clone(), b_next.clone())
+    for t, t0 in ((p, p0), (m, m0), (v, v0)):
+        t.copy_(t0)
+    gbar.zero_()
+    b_next.zero_()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            absnt.abs_normtest_adamw(grads, 0.1, 64, stats, gbar, b_next, p, m, v, HP, 4)
+            absnt.abs_adamw_step(p, gbar, m, v, HP, 5)
+    torch.cuda.current_stream().wait_stream(side)
+    for t, t0 in ((p, p0), (m, m0), (v, v0)):  # capture does not execute; start from the same state
+        t.copy_(t0)
+    graph.replay()
+    torch.cuda.synchronize()
+    got = (stats[:2], gbar, p, m, v, b_next)
+    for a, b in zip(got, want):
+        assert torch.equal(a, b)
+    assert int(b_next.item()) == ref["b_next"]
+
+
 # ------------------------------------------------------------------------- determinism
 def test_bit_identical_across_runs():
     K, d = 8, 3_000_017
