@@ -79,6 +79,44 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStre
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// The finalize kernel runs as one thread-block cluster.  The slice size (and with it the
+// shape of every sum) follows from the chunk counts alone; the cluster size only decides how
+// many warps share the slices.
+cudaError_t launch_finalize(FinalizeParams fp, cudaStream_t st) {
+  int slice = kFinalizeSlice;
+  for (;;) {
+    int64_t n = 0;
+    for (int s = 0; s < fp.n_shards; ++s)
+      n += (fp.chunk_prefix[s + 1] - fp.chunk_prefix[s] + slice - 1) / slice;
+    if (n <= kFinalizeMaxSlices) break;
+    slice *= 2;
+  }
+  fp.slice = slice;
+  fp.slice_prefix[0] = 0;
+  for (int s = 0; s < fp.n_shards; ++s)
+    fp.slice_prefix[s + 1] =
+        fp.slice_prefix[s] + (fp.chunk_prefix[s + 1] - fp.chunk_prefix[s] + slice - 1) / slice;
+  const int n_slices = fp.slice_prefix[fp.n_shards];
+  unsigned n_ctas = 1;
+  while (n_ctas < kFinalizeMaxCtas && static_cast<int>(n_ctas) * kFinalizeSlicesPerCta < n_slices)
+    n_ctas *= 2;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_ctas);
+  cfg.blockDim = dim3(kFinalizeThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = n_ctas;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, finalize_kernel, fp);
+}
+
 bool misaligned(const void* p, size_t a) {
   return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
 }
@@ -266,7 +304,7 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   fp.eta = eta;
   fp.norm = static_cast<double>(K);
   fp.b_cur = b_cur;
-  e = launch_pdl(finalize_kernel, dim3(1), dim3(kFinalizeThreads), st, fp);
+  e = launch_finalize(fp, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -414,7 +452,7 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
   fp.eta = eta;
   fp.norm = static_cast<double>(b - 1);
   fp.b_cur = b;
-  e = launch_pdl(finalize_kernel, dim3(1), dim3(kFinalizeThreads), st, fp);
+  e = launch_finalize(fp, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -566,7 +604,7 @@ extern "C" int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64
   fp.eta = eta;
   fp.norm = static_cast<double>(K);
   fp.b_cur = b_cur;
-  e = launch_pdl(finalize_kernel, dim3(1), dim3(kFinalizeThreads), st, fp);
+  e = launch_finalize(fp, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }

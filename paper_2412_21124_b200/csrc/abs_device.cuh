@@ -44,6 +44,8 @@ struct StreamParams {
 struct FinalizeParams {
   const double* chunk_in;
   int32_t chunk_prefix[ABS_MAX_SHARDS + 1];
+  int32_t slice_prefix[ABS_MAX_SHARDS + 1];  // slices of `slice` records before each shard
+  int slice;                                 // records per slice
   int n_shards;
   int n_chunks;
   double* stats; // header + shard records

@@ -18,6 +18,8 @@
 // their squares (and, in the unfused kernel, g_k^2) are fp32 over at most V*K terms per
 // thread-row, then accumulated in fp64.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "abs_device.cuh"
 
 namespace absnt {
@@ -387,91 +389,120 @@ __global__ void __launch_bounds__(kThreads, 2)
   }
 }
 
-// One CTA of kFinalizeThreads threads.  Shards with many chunks are reduced by the whole
-// CTA (thread t adds records t, t+T, ... in that order, four loads in flight, then a fixed
-// tree); shards with few chunks by one warp each.  Thread 0 then adds the shard records
-// in shard order, takes the decision (Algorithm 1: statistic T_k and the If/Else) and
-// writes the header.  The shape of every sum depends only on the chunk counts.
+// Finalize: one thread-block cluster of 1, 2, 4 or 8 CTAs x kFinalizeThreads threads.
+//
+// Every shard's chunk records are cut into slices of fp.slice consecutive records (a power of
+// two times 128, chosen by the host from the chunk counts alone so that at most
+// kFinalizeMaxSlices slices exist).  One warp reduces one slice: lane l adds records
+// l, l+32, ... of the slice in that order, four loads in flight, then a fixed shuffle tree;
+// slices go round-robin to the warps of the cluster, and each partial is stored into CTA 0's
+// shared memory (distributed shared memory for the other CTAs).  After the cluster barrier
+// (a hardware barrier between co-scheduled CTAs, not a spin on memory) CTA 0 adds, one warp
+// per shard, the shard's slice partials in lane-strided order and a tree, and its thread 0
+// adds the shard records in shard order, takes the decision (Algorithm 1: statistic T_k and
+// the If/Else) and writes the header.  The shape of every sum depends only on the chunk
+// counts, never on the number of CTAs or on which warp took which slice.
 constexpr int kFinalizeThreads = 1024;
 constexpr int kFinalizeWarps = kFinalizeThreads / 32;
-constexpr int kSmallShardChunks = 2048;
+constexpr int kFinalizeMaxCtas = 8;
+constexpr int kFinalizeSlice = 128;       // records: 32 lanes x 4 loads in flight
+constexpr int kFinalizeMaxSlices = 1024;  // 24 KB of partials in CTA 0
+constexpr int kFinalizeSlicesPerCta = 16;  // another CTA (another SM's L2 port) per 16 slices
 
-// records c0 + first, c0 + first + stride, ... (< c1), added in that order; eight loads in
-// flight per pass (absent records read as +0.0, which leaves the sums unchanged)
+// records c0 + first, c0 + first + stride, ... (< c1), added in that order.  Each pass issues
+// four unconditional loads (an index past the end re-reads the pass's first record and its
+// values are replaced by +0.0, which leaves the sums unchanged) before the first add.
 __device__ __forceinline__ void strided_records(const double* chunk_in, int c0, int c1, int first,
                                                 int stride, double& a, double& b, double& c) {
-  for (int ch = c0 + first; ch < c1; ch += 8 * stride) {
-    double2 t[16];
+  constexpr int kInFlight = 4;
+  for (int ch = c0 + first; ch < c1; ch += kInFlight * stride) {
+    double2 t[kInFlight];
+    double u2[kInFlight];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < kInFlight; ++u) {
       const int r = ch + u * stride;
-      if (r < c1) {
-        const double2* rec = reinterpret_cast<const double2*>(chunk_in + static_cast<int64_t>(r) * 4);
-        t[2 * u] = rec[0];
-        t[2 * u + 1] = rec[1];
-      } else {
-        t[2 * u] = make_double2(0.0, 0.0);
-        t[2 * u + 1] = make_double2(0.0, 0.0);
-      }
+      const double* rec = chunk_in + static_cast<int64_t>(r < c1 ? r : ch) * 4;
+      t[u] = __ldcg(reinterpret_cast<const double2*>(rec));
+      u2[u] = __ldcg(rec + 2);
     }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      a += t[2 * u].x;
-      b += t[2 * u].y;
-      c += t[2 * u + 1].x;
+    for (int u = 0; u < kInFlight; ++u) {
+      const bool live = ch + u * stride < c1;
+      a += live ? t[u].x : 0.0;
+      b += live ? t[u].y : 0.0;
+      c += live ? u2[u] : 0.0;
     }
+  }
+}
+
+__device__ __forceinline__ void warp_tree3(double& a, double& b, double& c) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    a += __shfl_down_sync(0xffffffffu, a, off);
+    b += __shfl_down_sync(0xffffffffu, b, off);
+    c += __shfl_down_sync(0xffffffffu, c, off);
   }
 }
 
 __global__ void __launch_bounds__(kFinalizeThreads)
     finalize_kernel(const __grid_constant__ FinalizeParams fp) {
-  __shared__ double red[kFinalizeWarps * 3];
+  namespace cg = cooperative_groups;
+  __shared__ double part[kFinalizeMaxSlices * 3];  // used in CTA 0 only
+  __shared__ double shard_tot[ABS_MAX_SHARDS * 3];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = static_cast<int>(cluster.block_rank());
+  const int n_warps = static_cast<int>(cluster.num_blocks()) * kFinalizeWarps;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double* part0 = cluster.map_shared_rank(part, 0);
+  const int n_slices = fp.slice_prefix[fp.n_shards];
   grid_dependency_wait();
-  // large shards: the whole CTA, one shard after the other
-  for (int s = 0; s < fp.n_shards; ++s) {
-    const int c0 = fp.chunk_prefix[s], c1 = fp.chunk_prefix[s + 1];
-    if (c1 - c0 <= kSmallShardChunks) continue;
-    double a = 0.0, b = 0.0, c = 0.0;
-    strided_records(fp.chunk_in, c0, c1, threadIdx.x, kFinalizeThreads, a, b, c);
-    block_reduce3<kFinalizeWarps>(a, b, c, red);
-    if (threadIdx.x == 0) {
-      double* rec = fp.stats + ABS_STATS_HEADER + s * ABS_SHARD_STRIDE;
-      rec[0] = a;
-      rec[1] = b;
-      rec[2] = c;
-      rec[3] = 0.0;
+  for (int i = rank * kFinalizeWarps + warp; i < n_slices; i += n_warps) {
+    // the shard of slice i: the last s with slice_prefix[s] <= i
+    int lo = 0, hi = fp.n_shards;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (fp.slice_prefix[mid] <= i) lo = mid; else hi = mid;
     }
-  }
-  // small shards: one warp per shard, round-robin
-  for (int s = warp; s < fp.n_shards; s += kFinalizeWarps) {
-    const int c0 = fp.chunk_prefix[s], c1 = fp.chunk_prefix[s + 1];
-    if (c1 - c0 > kSmallShardChunks) continue;
+    const int c0 = fp.chunk_prefix[lo] + (i - fp.slice_prefix[lo]) * fp.slice;
+    const int c1 = min(c0 + fp.slice, fp.chunk_prefix[lo + 1]);
     double a = 0.0, b = 0.0, c = 0.0;
     strided_records(fp.chunk_in, c0, c1, lane, 32, a, b, c);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      a += __shfl_down_sync(0xffffffffu, a, off);
-      b += __shfl_down_sync(0xffffffffu, b, off);
-      c += __shfl_down_sync(0xffffffffu, c, off);
+    warp_tree3(a, b, c);
+    if (lane == 0) {
+      part0[3 * i + 0] = a;
+      part0[3 * i + 1] = b;
+      part0[3 * i + 2] = c;
     }
+  }
+  // arrive.release / wait.acquire at cluster scope: every partial is visible to CTA 0
+  cluster.sync();
+  if (rank != 0) return;
+  for (int s = warp; s < fp.n_shards; s += kFinalizeWarps) {
+    double a = 0.0, b = 0.0, c = 0.0;
+    for (int i = fp.slice_prefix[s] + lane; i < fp.slice_prefix[s + 1]; i += 32) {
+      a += part[3 * i + 0];
+      b += part[3 * i + 1];
+      c += part[3 * i + 2];
+    }
+    warp_tree3(a, b, c);
     if (lane == 0) {
       double* rec = fp.stats + ABS_STATS_HEADER + s * ABS_SHARD_STRIDE;
       rec[0] = a;
       rec[1] = b;
       rec[2] = c;
       rec[3] = 0.0;
+      shard_tot[3 * s + 0] = a;
+      shard_tot[3 * s + 1] = b;
+      shard_tot[3 * s + 2] = c;
     }
   }
-  __threadfence_block();
   __syncthreads();
   if (threadIdx.x == 0) {
     double tot_n2 = 0.0, tot_S = 0.0, tot_Q = 0.0;
     for (int s = 0; s < fp.n_shards; ++s) {
-      const volatile double* rec = fp.stats + ABS_STATS_HEADER + s * ABS_SHARD_STRIDE;
-      tot_n2 += rec[0];
-      tot_S += rec[1];
-      tot_Q += rec[2];
+      tot_n2 += shard_tot[3 * s + 0];
+      tot_S += shard_tot[3 * s + 1];
+      tot_Q += shard_tot[3 * s + 2];
     }
     double T;
     int flags;
