@@ -229,6 +229,17 @@ def test_ragged_shards(dtype):
     assert got["shards"][2] == (0.0, 0.0, 0.0)
 
 
+def test_shards_spanning_several_record_slices():
+    # chunk counts 1, 128, 129, 0, 257 and a ragged rest: the final reduction cuts each shard's
+    # chunk records into slices of 128, so these sit on both sides of every slice boundary
+    c = 4096
+    offs = [0, c, 129 * c, 258 * c, 258 * c, 515 * c, 515 * c + 700 * c + 77]
+    d = offs[-1]
+    got, _ = run_and_check(2, d, torch.bfloat16, fused=True, seed=705, shard_offsets=offs)
+    assert got["n_chunks"] == 1 + 128 + 129 + 257 + 701
+    run_and_check(3, d, torch.float32, fused=False, seed=706, shard_offsets=offs)
+
+
 def test_equal_shards_and_max_shards():
     d = 100_000
     run_and_check(8, d, torch.bfloat16, fused=False, seed=710,
