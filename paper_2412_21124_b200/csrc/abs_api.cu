@@ -309,7 +309,31 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   return ABS_OK;
 }
 
-int persample_rows_per_block(int64_t b) { return b >= 2048 ? 128 : (b >= 512 ? 64 : 32); }
+// Rows per row block of the per-sample kernels: at most 512 (the row-block records then cost
+// 2% of the matrix traffic), and, while the grid is only a few waves of 148 SMs x 3 resident
+// CTAs, the count that fills whole waves (b=4096, d=16384: 13 row blocks x 32 column blocks =
+// 416 CTAs in one wave instead of 1024 in 2.3).  A function of (b, d) alone, so the shape of
+// every sum is too.
+int persample_rows_per_block(int64_t b, int64_t d) {
+  const int64_t wave = 148 * 3;
+  const int64_t col_blocks = ((d + 3) / 4 + kPsThreads - 1) / kPsThreads;
+  const int64_t nrb_min = (b + 511) / 512;
+  int64_t nrb = nrb_min;
+  if (nrb_min * col_blocks < 4 * wave) {
+    for (int64_t w = 1; w <= 4; ++w) {
+      nrb = w * wave / col_blocks;
+      if (nrb >= nrb_min) break;
+    }
+    if (nrb < nrb_min) nrb = nrb_min;
+  }
+  int64_t rpb = (b + nrb - 1) / nrb;
+  // whole register groups of kGroup rows while blocks are short (a ragged group costs a full one)
+  const int64_t q = rpb < 8 * kGroup ? kGroup : 4;
+  rpb = (rpb + q - 1) / q * q;
+  const int64_t grid_y_max = 65535;
+  if ((b + rpb - 1) / rpb > grid_y_max) rpb = (b + grid_y_max - 1) / grid_y_max;
+  return static_cast<int>(rpb < INT32_MAX ? rpb : INT32_MAX);
+}
 
 }  // namespace
 
@@ -325,7 +349,7 @@ size_t abs_stats_bytes(int64_t d, int n_shards) {
 
 size_t abs_persample_stats_bytes(int64_t b, int64_t d) {
   if (b < 2 || d < 1) return 0;
-  const int rpb = persample_rows_per_block(b);
+  const int rpb = persample_rows_per_block(b, d);
   const int64_t nrb = (b + rpb - 1) / rpb;
   const int64_t n_chunks = (d + kPsThreads - 1) / kPsThreads;
   return sizeof(double) *
@@ -404,7 +428,7 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
       misaligned(b_next_out, 8))
     return ABS_ERR_ALIGN;
   const int64_t n_chunks64 = (d + kPsThreads - 1) / kPsThreads;
-  const int rpb = persample_rows_per_block(b);
+  const int rpb = persample_rows_per_block(b, d);
   const int64_t nrb = (b + rpb - 1) / rpb;
   if (n_chunks64 > INT32_MAX || nrb > 65535) return ABS_ERR_RANGE;
 
