@@ -233,6 +233,46 @@ int64_t abs_decide(double S, double n2, double norm, double eta, int64_t b_cur, 
  * invalid arguments.  Host, pure. */
 int64_t abs_round_batch(int64_t b_next, int64_t J, int64_t M);
 
+/*
+ * The batch-size schedule around the test (Algorithm 1: the While loop's counters and the
+ * If branch; Sec. 5 "Training Specifications": a maximum global batch size above which the
+ * test is no longer performed, and a test interval; Tables 5-7: base and maximum micro batch
+ * size, base gradient accumulation steps).  Host-side integer state, no device work, no
+ * allocation; the caller owns the struct and may read its fields.
+ *
+ *   J          workers (data-parallel size)
+ *   M          gradient accumulation steps, grows when a new batch size needs a microbatch
+ *              above max_micro
+ *   micro      microbatch size b_{k,J}^M
+ *   b          global batch size b_k = J*M*micro
+ *   b_max      maximum global batch size
+ *   max_micro  maximum micro batch size, 0 = no limit (M then never changes)
+ *   interval   the test runs at steps k with k % interval == 0
+ *   step       k, starts at 1;  samples = i, the samples processed so far
+ *
+ * abs_schedule_advance(s, b_test) closes step k: b_test is the b_next the test wrote (pass
+ * s->b when no test ran).  With target = min(b_test, b_max):
+ *   target <= b:  nothing changes (the Else branch);
+ *   else          micro = ceil(target/(J*M));  if micro > max_micro > 0 then
+ *                 M = ceil(target/(J*max_micro)), micro = ceil(target/(J*M));  b = J*M*micro
+ *                 (the If branch); a b above b_max after rounding falls back to
+ *                 micro = floor(b_max/(J*M)), and is dropped if that does not exceed the old b.
+ * Then samples += the batch size step k used, step += 1.  The paper prints the rounding only;
+ * the growth rule for M and the fallback at the cap are this library's reading.
+ */
+typedef struct abs_schedule {
+  int64_t J, M, micro, b, b_max, max_micro, interval, step, samples;
+} abs_schedule;
+
+/* b = J*M*micro0 must not exceed b_max; micro0 must not exceed max_micro when that is set.
+ * Returns ABS_OK, ABS_ERR_NULL or ABS_ERR_RANGE (also when b_max exceeds 2^60). */
+int abs_schedule_init(abs_schedule* s, int64_t J, int64_t M, int64_t micro0, int64_t b_max,
+                      int64_t max_micro, int64_t interval);
+/* 1 if step s->step runs the test (b < b_max and step % interval == 0), else 0; -1 if s is NULL. */
+int abs_schedule_test_due(const abs_schedule* s);
+/* Returns ABS_OK, ABS_ERR_NULL, or ABS_ERR_RANGE (b_test < 1; the state is then unchanged). */
+int abs_schedule_advance(abs_schedule* s, int64_t b_test);
+
 const char* abs_status_string(int status);
 
 /* The cudaError_t of the most recent ABS_ERR_CUDA on this thread (0 if none). */

@@ -142,6 +142,49 @@ def round_batch(b_next, J, M):
     return int(lib().abs_oracle_round_batch(int(b_next), int(J), int(M)))
 
 
+class Schedule:
+    """Algorithm 1's loop state around the test, in Python integers (exact at any size): the
+    If branch (microbatch rounded up, minibatch = M * microbatch, global = J * minibatch), the
+    Else branch, and the counters k and i; with the maximum global batch size and test interval
+    of Sec. 5 ("Training Specifications") and the maximum micro batch size of Tables 5-7.  The
+    paper prints no rule for the last two beyond their values; the reading here is: when the
+    rounded microbatch would pass the maximum, M becomes the smallest count that keeps it
+    within the maximum; a batch that rounding pushes over the cap falls back to the largest
+    microbatch under the cap and is ignored if that is no increase."""
+
+    def __init__(self, J, M, micro0, b_max, max_micro=0, interval=1):
+        self.J, self.M, self.micro = J, M, micro0
+        self.b = J * M * micro0
+        self.b_max, self.max_micro, self.interval = b_max, max_micro, interval
+        self.step, self.samples = 1, 0
+        assert self.b <= b_max and (max_micro == 0 or micro0 <= max_micro)
+
+    def test_due(self):
+        return self.b < self.b_max and self.step % self.interval == 0
+
+    def advance(self, b_test):
+        used = self.b
+        target = min(b_test, self.b_max)
+        if target > self.b:
+            M = self.M
+            micro = -(-target // (self.J * M))
+            if self.max_micro and micro > self.max_micro:
+                M = -(-target // (self.J * self.max_micro))
+                micro = -(-target // (self.J * M))
+            b = self.J * M * micro
+            if b > self.b_max:
+                micro = self.b_max // (self.J * M)
+                b = self.J * M * micro
+            if micro >= 1 and b > self.b:
+                self.M, self.micro, self.b = M, micro, b
+        self.samples += used
+        self.step += 1
+
+    def state(self):
+        return dict(J=self.J, M=self.M, micro=self.micro, b=self.b, step=self.step,
+                    samples=self.samples)
+
+
 def adamw(w, m, v, g, lr, beta1, beta2, eps, wd, step):
     """w, m, v float32 arrays (the stored state), g float64; returns fp64 (w', m', v')."""
     w, m, v = (np.ascontiguousarray(x, dtype=np.float32) for x in (w, m, v))

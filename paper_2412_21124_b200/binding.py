@@ -76,6 +76,12 @@ def lib():
     L.abs_decide.argtypes = [dbl, dbl, dbl, dbl, i64, ptr, ptr]
     L.abs_round_batch.restype = i64
     L.abs_round_batch.argtypes = [i64, i64, i64]
+    L.abs_schedule_init.restype = cint
+    L.abs_schedule_init.argtypes = [ptr, i64, i64, i64, i64, i64, i64]
+    L.abs_schedule_test_due.restype = cint
+    L.abs_schedule_test_due.argtypes = [ptr]
+    L.abs_schedule_advance.restype = cint
+    L.abs_schedule_advance.argtypes = [ptr, i64]
     L.abs_status_string.restype = ctypes.c_char_p
     L.abs_status_string.argtypes = [cint]
     L.abs_last_cuda_error.restype = cint
@@ -297,6 +303,31 @@ def abs_decide(S, n2, norm, eta, b_cur):
 
 def abs_round_batch(b_next, J, M):
     return int(lib().abs_round_batch(int(b_next), int(J), int(M)))
+
+
+class AbsSchedule(ctypes.Structure):
+    """struct abs_schedule of the C header (host-side state of Algorithm 1's loop)."""
+    _fields_ = [(name, ctypes.c_int64) for name in
+                ("J", "M", "micro", "b", "b_max", "max_micro", "interval", "step", "samples")]
+
+
+def abs_schedule_init(J, M, micro0, b_max, max_micro=0, interval=1):
+    s = AbsSchedule()
+    rc = lib().abs_schedule_init(ctypes.byref(s), int(J), int(M), int(micro0), int(b_max),
+                                 int(max_micro), int(interval))
+    if rc != 0:
+        raise AbsError(rc, "abs_schedule_init")
+    return s
+
+
+def abs_schedule_test_due(s):
+    return bool(lib().abs_schedule_test_due(ctypes.byref(s)))
+
+
+def abs_schedule_advance(s, b_test):
+    rc = lib().abs_schedule_advance(ctypes.byref(s), int(b_test))
+    if rc != 0:
+        raise AbsError(rc, "abs_schedule_advance")
 
 
 def read_stats(stats_out, n_shards=1):

@@ -51,6 +51,10 @@ def test_header_is_plain_c_and_links_from_c(L, tmp_path):
         "  int rc = abs_adamw_step(0, 0, 0, 0, 10, &hp, 1, 0);\n"
         '  printf("%lld %.1f %d %lld %d %zu\\n", b, T, flags, (long long)abs_round_batch(259, 4, 16), rc,\n'
         "         abs_stats_bytes(1, 1));\n"
+        "  abs_schedule s;\n"
+        "  if (abs_schedule_init(&s, 4, 16, 4, 8192, 8, 1) != ABS_OK || !abs_schedule_test_due(&s)) return 1;\n"
+        "  if (abs_schedule_advance(&s, 1000) != ABS_OK) return 2;\n"
+        '  printf("%lld %lld %lld\\n", (long long)s.M, (long long)s.micro, (long long)s.b);\n'
         "  return 0;\n}\n")
     exe = tmp_path / "use_abi"
     lib_dir = os.path.dirname(binding._build.LIB_PATH)
@@ -58,7 +62,74 @@ def test_header_is_plain_c_and_links_from_c(L, tmp_path):
                            os.path.join(ROOT, "include"), str(src), "-o", str(exe), "-L", lib_dir,
                            "-labs_normtest", "-Wl,-rpath," + lib_dir])
     out = subprocess.check_output([str(exe)]).decode().split()
-    assert out == ["4", "4.0", "4", "320", str(binding.ABS_ERR_NULL), str(8 * 8 + 4 * 8 + 2 * 32)]
+    assert out == ["4", "4.0", "4", "320", str(binding.ABS_ERR_NULL), str(8 * 8 + 4 * 8 + 2 * 32),
+                   "32", "8", "1024"]
+
+
+def _sched_state(s):
+    return {k: getattr(s, k) for k in ("J", "M", "micro", "b", "step", "samples")}
+
+
+def test_schedule_hand_cases(L):
+    for c in json.load(open(GOLDEN))["schedule"]:
+        i = c["init"]
+        s = binding.abs_schedule_init(i["J"], i["M"], i["micro0"], i["b_max"], i["max_micro"],
+                                      i["interval"])
+        assert s.b == i["J"] * i["M"] * i["micro0"] and s.step == 1 and s.samples == 0
+        for st in c["steps"]:
+            assert binding.abs_schedule_test_due(s) == st["due"], c["name"]
+            binding.abs_schedule_advance(s, st["b_test"])
+            got = _sched_state(s)
+            assert {k: got[k] for k in st["after"]} == st["after"], c["name"]
+
+
+def test_schedule_matches_oracle_on_random_runs(L):
+    import numpy as np
+    from oracle import abs_oracle as orc
+    rng = np.random.default_rng(23)
+    for trial in range(100):
+        J, M, micro0 = int(rng.integers(1, 9)), int(rng.integers(1, 33)), int(rng.integers(1, 9))
+        max_micro = int(rng.integers(micro0, 4 * micro0 + 1)) if trial % 4 else 0
+        b_max = J * M * micro0 * int(rng.integers(1, 200)) + int(rng.integers(0, 50))
+        interval = int(rng.integers(1, 5))
+        s = binding.abs_schedule_init(J, M, micro0, b_max, max_micro, interval)
+        o = orc.Schedule(J, M, micro0, b_max, max_micro, interval)
+        for _ in range(40):
+            assert binding.abs_schedule_test_due(s) == o.test_due()
+            b_test = int(rng.integers(1, 3 * b_max)) if o.test_due() else o.b
+            binding.abs_schedule_advance(s, b_test)
+            o.advance(b_test)
+            assert _sched_state(s) == o.state()
+    # near the largest accepted cap: Python integers on one side, int64 on the other
+    big = 1 << 60
+    s = binding.abs_schedule_init(3, 5, 7, big, 11, 1)
+    o = orc.Schedule(3, 5, 7, big, 11, 1)
+    for b_test in (10**6, 10**12, big - 12345, big, 2**63 - 1):
+        binding.abs_schedule_advance(s, b_test)
+        o.advance(b_test)
+        assert _sched_state(s) == o.state()
+    assert s.b <= big and not binding.abs_schedule_test_due(s) == (s.b == big)
+
+
+def test_schedule_rejects(L):
+    s = binding.AbsSchedule()
+    ref = ctypes.byref(s)
+    assert L.abs_schedule_init(None, 4, 16, 4, 8192, 8, 1) == binding.ABS_ERR_NULL
+    for args in ((0, 16, 4, 8192, 8, 1), (4, 0, 4, 8192, 8, 1), (4, 16, 0, 8192, 8, 1),
+                 (4, 16, 4, 0, 8, 1), (4, 16, 4, 8192, -1, 1), (4, 16, 4, 8192, 8, 0),
+                 (4, 16, 4, 255, 8, 1),        # base batch 256 above the cap
+                 (4, 16, 9, 8192, 8, 1),       # base microbatch above its maximum
+                 (4, 16, 4, (1 << 60) + 1, 8, 1),
+                 (1 << 31, 1 << 31, 4, 1 << 60, 0, 1)):  # J*M*micro passes 2^60
+        assert L.abs_schedule_init(ref, *args) == binding.ABS_ERR_RANGE, args
+    assert L.abs_schedule_test_due(None) == -1
+    assert L.abs_schedule_advance(None, 5) == binding.ABS_ERR_NULL
+    assert L.abs_schedule_init(ref, 4, 16, 4, 8192, 8, 1) == 0
+    before = _sched_state(s)
+    assert L.abs_schedule_advance(ref, 0) == binding.ABS_ERR_RANGE
+    assert _sched_state(s) == before
+    with pytest.raises(binding.AbsError):
+        binding.abs_schedule_init(4, 16, 4, 255)
 
 
 def test_status_strings(L):
@@ -118,7 +189,8 @@ def test_stats_bytes(L):
     big = binding.abs_stats_bytes(124_439_808, 8)
     assert big % 16 == 0 and big < (1 << 20)
     assert binding.abs_persample_stats_bytes(1, 10) == 0
-    assert binding.abs_persample_stats_bytes(4096, 16384) > 3 * 32 * 16384 * 8
+    # three doubles per (row block, column), row blocks of at most 512 rows
+    assert binding.abs_persample_stats_bytes(4096, 16384) > 3 * (4096 // 512) * 16384 * 8
 
 
 # ---- invalid arguments: every path returns its status before any CUDA call ---------------

@@ -104,6 +104,67 @@ def test_round_batch_properties():
         assert r % (J * M) == 0 and b <= r < b + J * M
 
 
+def test_hand_case_schedule():
+    for c in json.load(open(GOLDEN))["schedule"]:
+        i = c["init"]
+        s = orc.Schedule(i["J"], i["M"], i["micro0"], i["b_max"], i["max_micro"], i["interval"])
+        for st in c["steps"]:
+            assert s.test_due() == st["due"], c["name"]
+            s.advance(st["b_test"])
+            got = s.state()
+            assert {k: got[k] for k in st["after"]} == st["after"], c["name"]
+
+
+def test_schedule_properties_and_brute_force_layout():
+    """Invariants of Algorithm 1's If/Else with the cap and the micro-batch limit, and the
+    layout checked against an exhaustive search on small numbers."""
+    rng = np.random.default_rng(11)
+    for trial in range(150):
+        J, M0, micro0 = int(rng.integers(1, 6)), int(rng.integers(1, 5)), int(rng.integers(1, 4))
+        max_micro = int(rng.integers(micro0, micro0 + 4)) if trial % 3 else 0
+        b0 = J * M0 * micro0
+        b_max = b0 + int(rng.integers(0, 400))
+        s = orc.Schedule(J, M0, micro0, b_max, max_micro, int(rng.integers(1, 4)))
+        total = 0
+        for k in range(1, 30):
+            before = s.state()
+            b_test = int(rng.integers(1, 2 * b_max))
+            s.advance(b_test)
+            after = s.state()
+            total += before["b"]
+            assert after["step"] == k + 1 and after["samples"] == total
+            assert after["b"] == J * after["M"] * after["micro"]
+            assert before["b"] <= after["b"] <= b_max            # never shrinks, never passes the cap
+            assert max_micro == 0 or after["micro"] <= max_micro
+            assert after["M"] >= before["M"] and (max_micro or after["M"] == M0)
+            target = min(b_test, b_max)
+            if target <= before["b"]:
+                assert after == dict(before, step=k + 1, samples=total)  # Else branch
+                continue
+            # If branch: among layouts (M', micro') allowed by the limit, with M' the paper's M
+            # when its rounded microbatch fits and otherwise the smallest M' that fits, the
+            # batch is the smallest J*M'*micro' >= target; found here by exhaustive search
+            M_fit = None
+            for Mc in range(before["M"], b_max + 1):
+                mic = -(-target // (J * Mc))
+                if max_micro == 0 or mic <= max_micro:
+                    M_fit = (Mc, mic)
+                    break
+            Mc, mic = M_fit
+            want = J * Mc * mic
+            if want <= b_max:
+                assert (after["M"], after["micro"], after["b"]) == (Mc, mic, want)
+                assert target <= after["b"] < target + J * Mc
+                if Mc == before["M"]:
+                    assert after["b"] == orc.round_batch(target, J, before["M"])
+            else:  # rounding passed the cap: largest multiple of J*Mc under it, if an increase
+                fb = (b_max // (J * Mc)) * J * Mc
+                if fb > before["b"]:
+                    assert after["b"] == fb and after["M"] == Mc
+                else:
+                    assert after["b"] == before["b"] and after["M"] == before["M"]
+
+
 # ------------------------------------------------------------- exact rational brute force
 @pytest.mark.parametrize("K,d", [(1, 1), (2, 3), (3, 5), (4, 8), (5, 7), (7, 2)])
 @pytest.mark.parametrize("kind", ["f32", "bf16"])
