@@ -503,7 +503,11 @@ def persample_check(G, eta):
 @pytest.mark.parametrize("b,d,ld,shift", [(2, 5, 5, 0), (7, 4100, 4100, 0), (32, 1000, 1000, 0),
                                           (33, 300, 320, 0), (100, 2051, 2052, 1),
                                           (257, 4096, 4096, 0), (1000, 777, 800, 0),
-                                          (2049, 515, 516, 0)])
+                                          (2049, 515, 516, 0),
+                                          (130, 700, 700, 0),      # few rows per row block
+                                          (4096, 1000, 1000, 0),   # narrow and tall: many row blocks
+                                          (1500, 300, 304, 2),     # the same, rows misaligned, ragged last block
+                                          (65, 40_000, 40_000, 0)])
 def test_persample_shapes(b, d, ld, shift):
     gen = torch.Generator(device=DEV)
     gen.manual_seed(b * 131 + d)
@@ -543,13 +547,17 @@ def test_least_squares_schedule_step_locked(eta):
     v = torch.zeros_like(w)
     gbar = torch.empty(d, dtype=torch.float32, device=DEV)
     b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
-    b, traj, checked = 32, [], 0
+    sched = absnt.abs_schedule_init(1, 1, 32, b_max)  # J = M = 1: the microbatch is the batch
+    traj, checked = [], 0
     for t in range(steps):
+        b = int(sched.b)
+        assert int(sched.step) == t + 1
         x, y = synth.lsq_batch(b, w_star, 1500, t)
         G = synth.lsq_persample_grads(x, y, w)
         stats = absnt.alloc_persample_stats(b, d, DEV)
         absnt.abs_persample_norm_test(G, eta, stats, gbar, b_next)
-        testing = b < b_max
+        testing = absnt.abs_schedule_test_due(sched)
+        assert testing == (b < b_max)
         if testing or t % 40 == 0:
             ref = orc.persample(G.cpu().numpy(), eta)
             got = absnt.read_stats(stats)
@@ -569,8 +577,9 @@ def test_least_squares_schedule_step_locked(eta):
             assert_vec_close(m, m_ref, "m")
             assert_vec_close(v, v_ref, "v")
         traj.append(b)
-        if testing:
-            b = min(int(b_next.item()), b_max)  # the paper's device->host crossing
+        # the paper's device->host crossing, once per tested step
+        absnt.abs_schedule_advance(sched, int(b_next.item()) if testing else b)
+    assert int(sched.samples) == sum(traj)
     assert traj[0] == 32 and traj[-1] == b_max
     assert all(a <= c for a, c in zip(traj, traj[1:]))  # never decreases
     assert checked >= 5
