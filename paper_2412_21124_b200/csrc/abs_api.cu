@@ -327,9 +327,8 @@ int persample_rows_per_block(int64_t b, int64_t d) {
     if (nrb < nrb_min) nrb = nrb_min;
   }
   int64_t rpb = (b + nrb - 1) / nrb;
-  // whole register groups of kGroup rows while blocks are short (a ragged group costs a full one)
-  const int64_t q = rpb < 8 * kGroup ? kGroup : 4;
-  rpb = (rpb + q - 1) / q * q;
+  // whole groups of kGroup rows (only the last row block ends in a ragged group)
+  rpb = (rpb + kGroup - 1) / kGroup * kGroup;
   const int64_t grid_y_max = 65535;
   if ((b + rpb - 1) / rpb > grid_y_max) rpb = (b + grid_y_max - 1) / grid_y_max;
   return static_cast<int>(rpb < INT32_MAX ? rpb : INT32_MAX);

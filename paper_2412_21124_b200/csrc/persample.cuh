@@ -3,11 +3,16 @@
 // are per-sample gradients, reading the matrix once.
 //
 // Pass 1 (2-D grid: column block x row block): a thread owns VC adjacent columns and
-// walks its row block in groups of kGroup rows held in registers.  Per group and
-// column it forms the group mean (fp64 sum) and the within-group squared deviations
-// (fp32), and merges them into running {mean, M2} with the pairwise update
+// walks its row block in groups of kGroup rows.  Each value is consumed once, as it arrives:
+// per group and column the thread accumulates sum(x) in fp64 and, about a centre c close to
+// the column mean (the first row for the first group, the running mean afterwards),
+// sum((x-c)^2) in fp32; then
+//     mu_g = sum(x)/n_g,   M2_g = sum((x-c)^2) - n_g (mu_g-c)^2        (shift identity)
+// and the group is merged into the running {mean, M2} with the pairwise update
 //     delta = mu_g - mean;  mean += delta*n_g/(n+n_g);  M2 += M2_g + delta^2*n*n_g/(n+n_g)
-// (law of total variance).  It writes {mean, M2, Q} per (row block, column).
+// (law of total variance).  Because no value is needed twice, the rows are loaded in half
+// groups, the next half in flight while the current one is consumed.  It writes
+// {mean, M2, Q} per (row block, column).
 // Pass 2 (one thread per column): merges the row blocks in index order with the same
 // update, writes gbar, and reduces {gbar^2, M2, Q} over 128-column chunks for the
 // shared finalize kernel.
@@ -17,7 +22,8 @@
 
 namespace absnt {
 
-constexpr int kGroup = 16;      // rows held in registers at a time
+constexpr int kGroup = 16;      // rows per group (one shift centre, one merge)
+constexpr int kHalf = kGroup / 2; // rows per load batch
 constexpr int kPsThreads = 128; // threads per CTA of the per-sample kernels
 
 struct PersampleParams {
@@ -32,6 +38,57 @@ struct PersampleParams {
   double* chunk_out; // 4 doubles per kPsThreads-column chunk
 };
 
+// rows r .. r+kHalf-1 of this thread's columns; rows at or past r_end read as zero
+template <int VC, bool FULL>
+__device__ __forceinline__ void ps_load_half(const PersampleParams& prm, int64_t r, int64_t r_end,
+                                             int64_t c0, bool vec_cols, float (&x)[kHalf][VC]) {
+#pragma unroll
+  for (int j = 0; j < kHalf; ++j) {
+    const float* row = prm.G + (r + j) * prm.ld + c0;
+    if (FULL || r + j < r_end) {
+      if (VC == 4 && vec_cols) {
+        const uint4 t = ld_once_16(row);
+        x[j][0] = __uint_as_float(t.x);
+        x[j][1 % VC] = __uint_as_float(t.y);
+        x[j][2 % VC] = __uint_as_float(t.z);
+        x[j][3 % VC] = __uint_as_float(t.w);
+      } else {
+#pragma unroll
+        for (int i = 0; i < VC; ++i) x[j][i] = (c0 + i < prm.d) ? __ldg(row + i) : 0.f;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < VC; ++i) x[j][i] = 0.f;
+    }
+  }
+}
+
+// Accumulators of one group: sum(x) in two fp64 chains (even and odd rows), the shifted
+// squares and the plain squares in fp32.
+template <int VC>
+struct PsGroup {
+  double s0[VC], s1[VC];
+  float c[VC], s2[VC], q[VC];
+};
+
+template <int VC, bool FULL>
+__device__ __forceinline__ void ps_consume_half(PsGroup<VC>& g, const float (&x)[kHalf][VC],
+                                                int n_live) {
+#pragma unroll
+  for (int j = 0; j < kHalf; ++j) {
+    if (FULL || j < n_live) {
+#pragma unroll
+      for (int i = 0; i < VC; ++i) {
+        const float v = x[j][i];
+        if (j & 1) g.s1[i] += static_cast<double>(v); else g.s0[i] += static_cast<double>(v);
+        const float dv = v - g.c[i];
+        g.s2[i] = fmaf(dv, dv, g.s2[i]);
+        g.q[i] = fmaf(v, v, g.q[i]);
+      }
+    }
+  }
+}
+
 template <int VC>
 __global__ void __launch_bounds__(kPsThreads, 3)
     persample_partial_kernel(const __grid_constant__ PersampleParams prm) {
@@ -40,61 +97,65 @@ __global__ void __launch_bounds__(kPsThreads, 3)
   if (c0 >= prm.d) return;
   const int64_t r0 = static_cast<int64_t>(blockIdx.y) * prm.rows_per_block;
   const int64_t r1 = (r0 + prm.rows_per_block < prm.b) ? r0 + prm.rows_per_block : prm.b;
-  const bool full_cols = (c0 + VC <= prm.d);
+  const bool vec_cols = (c0 + VC <= prm.d);
 
   double mean[VC], m2[VC], qq[VC];
 #pragma unroll
   for (int i = 0; i < VC; ++i) mean[i] = m2[i] = qq[i] = 0.0;
-  int n = 0;
+  int64_t n = 0;
+  PsGroup<VC> g;
+  float xa[kHalf][VC], xb[kHalf][VC];
 
-  for (int64_t r = r0; r < r1; r += kGroup) {
-    const int ng = (r1 - r < kGroup) ? static_cast<int>(r1 - r) : kGroup;
-    float x[kGroup][VC];
+  // centre of the next group and cleared accumulators; `first` = first row of the group
+  auto open_group = [&](const float (&first)[VC]) {
 #pragma unroll
-    for (int j = 0; j < kGroup; ++j) {
-      const float* row = prm.G + (r + j) * prm.ld + c0;
-      if (j < ng) {
-        if (VC == 4 && full_cols) {
-          const uint4 t = ld_once_16(row);
-          x[j][0] = __uint_as_float(t.x);
-          x[j][1 % VC] = __uint_as_float(t.y);
-          x[j][2 % VC] = __uint_as_float(t.z);
-          x[j][3 % VC] = __uint_as_float(t.w);
-        } else {
-#pragma unroll
-          for (int i = 0; i < VC; ++i) x[j][i] = (c0 + i < prm.d) ? __ldg(row + i) : 0.f;
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < VC; ++i) x[j][i] = 0.f;
-      }
+    for (int i = 0; i < VC; ++i) {
+      g.c[i] = (n == 0) ? first[i] : static_cast<float>(mean[i]);
+      g.s0[i] = g.s1[i] = 0.0;
+      g.s2[i] = g.q[i] = 0.f;
     }
-    const double inv_ng = 1.0 / static_cast<double>(ng);
+  };
+  auto close_group = [&](int ng) {
+    const double dn = static_cast<double>(ng);
     const double nn = static_cast<double>(n + ng);
-    const double w_mean = static_cast<double>(ng) / nn;
+    const double w_mean = dn / nn;
     const double w_m2 = static_cast<double>(n) * w_mean;
 #pragma unroll
     for (int i = 0; i < VC; ++i) {
-      double s = 0.0;
-#pragma unroll
-      for (int j = 0; j < kGroup; ++j) s += static_cast<double>(x[j][i]); // absent rows are 0
-      const double mu = s * inv_ng;
-      const float muf = static_cast<float>(mu);
-      float dev2 = 0.f, sq = 0.f;
-#pragma unroll
-      for (int j = 0; j < kGroup; ++j) {
-        if (j < ng) {
-          const float dv = x[j][i] - muf;
-          dev2 = fmaf(dv, dv, dev2);
-          sq = fmaf(x[j][i], x[j][i], sq);
-        }
-      }
+      const double sum = g.s0[i] + g.s1[i];
+      // a power-of-two count divides exactly by multiplication; a ragged count by division,
+      // so that identical rows give their common value exactly
+      const double mu = (ng == kGroup) ? sum * (1.0 / kGroup) : sum / dn;
+      const double dc = mu - static_cast<double>(g.c[i]);
+      const double m2g = fmax(static_cast<double>(g.s2[i]) - dn * dc * dc, 0.0);
       const double delta = mu - mean[i];
       mean[i] += delta * w_mean;
-      m2[i] += static_cast<double>(dev2) + delta * delta * w_m2;
-      qq[i] += static_cast<double>(sq);
+      m2[i] += m2g + delta * delta * w_m2;
+      qq[i] += static_cast<double>(g.q[i]);
     }
     n += ng;
+  };
+
+  const int64_t n_full = (r1 - r0) / kGroup;
+  int64_t r = r0;
+  if (n_full > 0) ps_load_half<VC, true>(prm, r, r1, c0, vec_cols, xa);
+  for (int64_t gi = 0; gi < n_full; ++gi) {
+    open_group(xa[0]);
+    ps_load_half<VC, true>(prm, r + kHalf, r1, c0, vec_cols, xb);
+    ps_consume_half<VC, true>(g, xa, kHalf);
+    if (gi + 1 < n_full) ps_load_half<VC, true>(prm, r + kGroup, r1, c0, vec_cols, xa);
+    ps_consume_half<VC, true>(g, xb, kHalf);
+    close_group(kGroup);
+    r += kGroup;
+  }
+  if (r < r1) {  // the last, ragged group of the row block
+    const int ng = static_cast<int>(r1 - r);
+    ps_load_half<VC, false>(prm, r, r1, c0, vec_cols, xa);
+    ps_load_half<VC, false>(prm, r + kHalf, r1, c0, vec_cols, xb);
+    open_group(xa[0]);
+    ps_consume_half<VC, false>(g, xa, ng);
+    ps_consume_half<VC, false>(g, xb, ng - kHalf);
+    close_group(ng);
   }
   const int64_t o = static_cast<int64_t>(blockIdx.y) * prm.d + c0;
 #pragma unroll
