@@ -234,6 +234,28 @@ int64_t abs_decide(double S, double n2, double norm, double eta, int64_t b_cur, 
 int64_t abs_round_batch(int64_t b_next, int64_t J, int64_t M);
 
 /*
+ * Mixed precision (Sec. 5: the experiments train in bfloat16): the two update calls with one
+ * more output, a bfloat16 copy of the updated parameters -- the working copy the next
+ * forward pass reads while `params` stays the fp32 master -- written in the same pass
+ * (+2 B per coordinate instead of a separate 6 B cast pass).  Each bf16 value is the fp32
+ * value stored to `params`, rounded to nearest, ties to even.
+ *   params_bf16_out  device, d 16-bit elements, 2-byte aligned (16-byte alignment keeps the
+ *                    vector path); must not alias another argument
+ * abs_normtest_adamw_mixed: all other arguments as abs_normtest_adamw.
+ * abs_adamw_step_mixed: as abs_adamw_step; with stats_in non-NULL the gradient is clipped as
+ * in abs_adamw_step_clipped (max_norm finite, > 0), with stats_in NULL max_norm is ignored.
+ */
+int abs_normtest_adamw_mixed(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                             const int64_t* shard_offsets, int n_shards, double eta,
+                             int64_t b_cur, void* stats_out, float* gbar_out, int64_t* b_next_out,
+                             float* params, float* m, float* v, void* params_bf16_out,
+                             const abs_adamw_hparams* hparams, int64_t step, abs_stream_t stream);
+int abs_adamw_step_mixed(float* params, const float* gbar, float* m, float* v,
+                         void* params_bf16_out, int64_t d, const abs_adamw_hparams* hparams,
+                         int64_t step, double max_norm, const void* stats_in,
+                         abs_stream_t stream);
+
+/*
  * The batch-size schedule around the test (Algorithm 1: the While loop's counters and the
  * If branch; Sec. 5 "Training Specifications": a maximum global batch size above which the
  * test is no longer performed, and a test interval; Tables 5-7: base and maximum micro batch

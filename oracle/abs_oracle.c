@@ -30,6 +30,8 @@
  *                          the b_{k+1} display after Eq. 3).
  *   abs_oracle_adamw       the AdamW lines of Algorithm 1.
  *   abs_oracle_round_batch the three rounding lines of Algorithm 1's If branch.
+ *   abs_oracle_bf16_round  the bfloat16 working copy of fp32 parameters (Sec. 5: bfloat16
+ *                          training): round to nearest even.
  *   abs_oracle_clip_scale  global-norm gradient clipping as used in the paper's experiments
  *                          (Sec. 5 "gradient clipping"; "Gradient clipping 1.0" in the
  *                          hyper-parameter tables of Appendix C).  The paper gives no formula;
@@ -293,6 +295,47 @@ int abs_oracle_adamw(const float* w, const float* m, const float* v, const doubl
 double abs_oracle_clip_scale(double n2, double max_norm) {
   const double coef = max_norm / (sqrt(n2) + 1e-6);
   return coef < 1.0 ? coef : 1.0;
+}
+
+/*
+ * bfloat16 copy of fp32 values for mixed-precision training (Sec. 5: the experiments run in
+ * bfloat16): round to nearest, ties to even, written as the definition.  A bfloat16 is an fp32
+ * whose low 16 bits are zero; the two candidates are x with those bits cleared (toward zero)
+ * and the next such value away from zero; the nearer one wins (distances exact in fp64), a tie
+ * goes to the candidate whose last kept bit is 0.  Past the largest finite bfloat16 the
+ * away-from-zero candidate counts as 2^128 and yields infinity (IEEE 754 overflow rule).
+ * NaN maps to a quiet NaN with the input's sign and high payload bits.
+ */
+int abs_oracle_bf16_round(const float* x, int64_t n, uint16_t* out) {
+  if (!x || !out || n < 0) return -1;
+  for (int64_t i = 0; i < n; ++i) {
+    uint32_t bits;
+    memcpy(&bits, &x[i], 4);
+    if (x[i] != x[i]) {
+      out[i] = (uint16_t)((bits >> 16) | 0x0040u);
+      continue;
+    }
+    const uint32_t lo_bits = bits & 0xFFFF0000u;
+    const uint32_t hi_bits = lo_bits + 0x00010000u;
+    float lo_f, hi_f;
+    memcpy(&lo_f, &lo_bits, 4);
+    memcpy(&hi_f, &hi_bits, 4);
+    const double dx = (double)x[i];
+    const double dlo = (double)lo_f;
+    double dhi = (double)hi_f;
+    if (isinf(hi_f) && !isinf(x[i])) dhi = copysign(ldexp(1.0, 128), dx);
+    if (isinf(x[i])) {
+      out[i] = (uint16_t)(bits >> 16);
+      continue;
+    }
+    const double a = fabs(dx - dlo), b = fabs(dhi - dx);
+    uint32_t pick;
+    if (a < b) pick = lo_bits;
+    else if (b < a) pick = hi_bits;
+    else pick = ((lo_bits >> 16) & 1u) ? hi_bits : lo_bits;
+    out[i] = (uint16_t)(pick >> 16);
+  }
+  return 0;
 }
 
 /* AdamW on the clipped gradient scale*g (scale from abs_oracle_clip_scale). */

@@ -54,6 +54,8 @@ def lib():
         L.abs_oracle_adamw.restype = cint
         L.abs_oracle_adamw.argtypes = [ptr, ptr, ptr, ptr, i64, dbl, dbl, dbl, dbl, dbl, i64,
                                        ptr, ptr, ptr]
+        L.abs_oracle_bf16_round.restype = cint
+        L.abs_oracle_bf16_round.argtypes = [ptr, i64, ptr]
         L.abs_oracle_clip_scale.restype = dbl
         L.abs_oracle_clip_scale.argtypes = [dbl, dbl]
         L.abs_oracle_adamw_clipped.restype = cint
@@ -198,6 +200,15 @@ def adamw(w, m, v, g, lr, beta1, beta2, eps, wd, step):
     if rc != 0:
         raise ValueError("abs_oracle_adamw rejected its arguments")
     return wo, mo, vo
+
+
+def bf16_round(x):
+    """float32 array -> uint16 array of bfloat16 bit patterns, round to nearest even."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint16)
+    if lib().abs_oracle_bf16_round(_p(x), int(x.size), _p(out)) != 0:
+        raise ValueError("abs_oracle_bf16_round rejected its arguments")
+    return out
 
 
 def clip_scale(n2, max_norm):

@@ -70,6 +70,11 @@ def lib():
                                      ptr, ptr, ptr, ptr, i64, ptr]
     L.abs_normtest_adamw_noalloc.restype = cint
     L.abs_normtest_adamw_noalloc.argtypes = list(L.abs_normtest_adamw.argtypes)
+    L.abs_normtest_adamw_mixed.restype = cint
+    L.abs_normtest_adamw_mixed.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64, ptr, ptr,
+                                           ptr, ptr, ptr, ptr, ptr, ptr, i64, ptr]
+    L.abs_adamw_step_mixed.restype = cint
+    L.abs_adamw_step_mixed.argtypes = [ptr, ptr, ptr, ptr, ptr, i64, ptr, i64, dbl, ptr, ptr]
     L.abs_persample_norm_test.restype = cint
     L.abs_persample_norm_test.argtypes = [ptr, i64, i64, i64, cint, dbl, ptr, ptr, ptr, ptr]
     L.abs_decide.restype = i64
@@ -219,6 +224,52 @@ def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, param
                                   v.data_ptr(), ctypes.byref(hp), int(step), _stream(stream))
     if rc != ABS_OK:
         raise AbsError(rc, "abs_normtest_adamw")
+
+
+def _check_bf16_vec(t, d, name):
+    if t.dtype != torch.bfloat16 or t.dim() != 1 or t.numel() != d or t.stride(0) != 1:
+        raise TypeError("%s must be a contiguous bfloat16 vector of %d elements" % (name, d))
+    if not t.is_cuda:
+        raise TypeError("%s must live on a CUDA device" % name)
+
+
+def abs_normtest_adamw_mixed(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v,
+                             params_bf16_out, hparams, step, shard_offsets=None, stream=None):
+    """abs_normtest_adamw that also writes a bfloat16 copy of the updated parameters."""
+    table, K, d, code = _grad_table(grads)
+    offs, n_shards = _offsets(shard_offsets)
+    for t, name in ((params, "params"), (m, "m"), (v, "v")):
+        _check_f32_vec(t, d, name)
+    _check_bf16_vec(params_bf16_out, d, "params_bf16_out")
+    if gbar_out is not None:
+        _check_f32_vec(gbar_out, d, "gbar_out")
+    hp = _hparams(hparams)
+    rc = lib().abs_normtest_adamw_mixed(table, K, d, code, offs, n_shards, float(eta),
+                                        int(b_cur), stats_out.data_ptr(),
+                                        gbar_out.data_ptr() if gbar_out is not None else None,
+                                        b_next_out.data_ptr(), params.data_ptr(), m.data_ptr(),
+                                        v.data_ptr(), params_bf16_out.data_ptr(),
+                                        ctypes.byref(hp), int(step), _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_normtest_adamw_mixed")
+
+
+def abs_adamw_step_mixed(params, gbar, m, v, params_bf16_out, hparams, step, max_norm=0.0,
+                         stats_in=None, stream=None):
+    """abs_adamw_step (clipped to max_norm when stats_in is given) that also writes a bfloat16
+    copy of the updated parameters."""
+    d = params.numel()
+    for t, name in ((params, "params"), (gbar, "gbar"), (m, "m"), (v, "v")):
+        _check_f32_vec(t, d, name)
+    _check_bf16_vec(params_bf16_out, d, "params_bf16_out")
+    hp = _hparams(hparams)
+    rc = lib().abs_adamw_step_mixed(params.data_ptr(), gbar.data_ptr(), m.data_ptr(),
+                                    v.data_ptr(), params_bf16_out.data_ptr(), d,
+                                    ctypes.byref(hp), int(step), float(max_norm),
+                                    stats_in.data_ptr() if stats_in is not None else None,
+                                    _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_adamw_step_mixed")
 
 
 def abs_normtest_adamw_noalloc(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v,

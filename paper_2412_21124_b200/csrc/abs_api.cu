@@ -235,8 +235,8 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
 int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                   const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
                   void* stats_out, float* gbar_out, int64_t* b_next_out, float* params, float* m,
-                  float* v, const abs_adamw_hparams* hparams, int64_t step, bool fused,
-                  abs_stream_t stream) {
+                  float* v, void* params_bf16, const abs_adamw_hparams* hparams, int64_t step,
+                  bool fused, abs_stream_t stream) {
   if (!grads || !stats_out || !b_next_out) return ABS_ERR_NULL;
   if (!fused && !gbar_out) return ABS_ERR_NULL;
   if (fused && (!params || !m || !v)) return ABS_ERR_NULL;
@@ -256,6 +256,7 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   if (gbar_out && misaligned(gbar_out, 4)) return ABS_ERR_ALIGN;
   if (fused && (misaligned(params, 4) || misaligned(m, 4) || misaligned(v, 4)))
     return ABS_ERR_ALIGN;
+  if (params_bf16 && misaligned(params_bf16, 2)) return ABS_ERR_ALIGN;
 
   Layout L;
   const int rc = make_layout(d, shard_offsets, n_shards, fused, &L);
@@ -282,6 +283,7 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   prm.p = params;
   prm.m = m;
   prm.v = v;
+  prm.p16 = static_cast<uint16_t*>(params_bf16);
   prm.chunk_out = chunk_out;
   if (fused) prm.adam = make_adam(hparams, step);
 
@@ -360,7 +362,8 @@ int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                   const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
                   void* stats_out, float* gbar_out, int64_t* b_next_out, abs_stream_t stream) {
   return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
-                       gbar_out, b_next_out, nullptr, nullptr, nullptr, nullptr, 0, false, stream);
+                       gbar_out, b_next_out, nullptr, nullptr, nullptr, nullptr, nullptr, 0, false,
+                       stream);
 }
 
 int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dtype,
@@ -369,22 +372,35 @@ int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dty
                        float* m, float* v, const abs_adamw_hparams* hparams, int64_t step,
                        abs_stream_t stream) {
   return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
-                       gbar_out, b_next_out, params, m, v, hparams, step, true, stream);
+                       gbar_out, b_next_out, params, m, v, nullptr, hparams, step, true, stream);
+}
+
+int abs_normtest_adamw_mixed(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                             const int64_t* shard_offsets, int n_shards, double eta,
+                             int64_t b_cur, void* stats_out, float* gbar_out, int64_t* b_next_out,
+                             float* params, float* m, float* v, void* params_bf16_out,
+                             const abs_adamw_hparams* hparams, int64_t step, abs_stream_t stream) {
+  if (!params_bf16_out) return ABS_ERR_NULL;
+  return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
+                       gbar_out, b_next_out, params, m, v, params_bf16_out, hparams, step, true,
+                       stream);
 }
 
 namespace {
 int run_adamw(float* params, const float* gbar, float* m, float* v, int64_t d,
               const abs_adamw_hparams* hparams, int64_t step, const double* n2_dev,
-              double max_norm, abs_stream_t stream) {
+              double max_norm, void* params_bf16, abs_stream_t stream) {
   if (!params || !gbar || !m || !v) return ABS_ERR_NULL;
   if (d < 1) return ABS_ERR_RANGE;
   const int rc = check_hparams(hparams, step);
   if (rc != ABS_OK) return rc;
   if (misaligned(params, 4) || misaligned(gbar, 4) || misaligned(m, 4) || misaligned(v, 4))
     return ABS_ERR_ALIGN;
+  if (params_bf16 && misaligned(params_bf16, 2)) return ABS_ERR_ALIGN;
+  uint16_t* p16 = static_cast<uint16_t*>(params_bf16);
   const AdamScalars a = make_adam(hparams, step);
   const bool vec = !(misaligned(params, 16) || misaligned(gbar, 16) || misaligned(m, 16) ||
-                     misaligned(v, 16));
+                     misaligned(v, 16) || (p16 && misaligned(p16, 8)));
   // one CTA per 2048 vectors (two per thread), so CTAs retire and are replaced
   // continuously, as in the streaming kernels; a grid-stride loop covers huge d
   const int64_t work = vec ? (d + 3) / 4 : d;
@@ -394,8 +410,10 @@ int run_adamw(float* params, const float* gbar, float* m, float* v, int64_t d,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid(static_cast<unsigned>(blocks)), block(kThreads);
   const cudaError_t e =
-      vec ? launch_pdl(adamw_kernel<true>, grid, block, st, params, gbar, m, v, d, a, n2_dev, max_norm)
-          : launch_pdl(adamw_kernel<false>, grid, block, st, params, gbar, m, v, d, a, n2_dev, max_norm);
+      vec ? launch_pdl(adamw_kernel<true>, grid, block, st, params, gbar, m, v, d, a, n2_dev,
+                       max_norm, p16)
+          : launch_pdl(adamw_kernel<false>, grid, block, st, params, gbar, m, v, d, a, n2_dev,
+                       max_norm, p16);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -403,7 +421,7 @@ int run_adamw(float* params, const float* gbar, float* m, float* v, int64_t d,
 
 int abs_adamw_step(float* params, const float* gbar, float* m, float* v, int64_t d,
                    const abs_adamw_hparams* hparams, int64_t step, abs_stream_t stream) {
-  return run_adamw(params, gbar, m, v, d, hparams, step, nullptr, 0.0, stream);
+  return run_adamw(params, gbar, m, v, d, hparams, step, nullptr, 0.0, nullptr, stream);
 }
 
 int abs_adamw_step_clipped(float* params, const float* gbar, float* m, float* v, int64_t d,
@@ -413,7 +431,22 @@ int abs_adamw_step_clipped(float* params, const float* gbar, float* m, float* v,
   if (!std::isfinite(max_norm) || !(max_norm > 0.0)) return ABS_ERR_RANGE;
   if (misaligned(stats_in, 8)) return ABS_ERR_ALIGN;
   return run_adamw(params, gbar, m, v, d, hparams, step,
-                   static_cast<const double*>(stats_in) + ABS_STAT_N2, max_norm, stream);
+                   static_cast<const double*>(stats_in) + ABS_STAT_N2, max_norm, nullptr, stream);
+}
+
+int abs_adamw_step_mixed(float* params, const float* gbar, float* m, float* v,
+                         void* params_bf16_out, int64_t d, const abs_adamw_hparams* hparams,
+                         int64_t step, double max_norm, const void* stats_in,
+                         abs_stream_t stream) {
+  if (!params_bf16_out) return ABS_ERR_NULL;
+  const double* n2_dev = nullptr;
+  if (stats_in) {
+    if (!std::isfinite(max_norm) || !(max_norm > 0.0)) return ABS_ERR_RANGE;
+    if (misaligned(stats_in, 8)) return ABS_ERR_ALIGN;
+    n2_dev = static_cast<const double*>(stats_in) + ABS_STAT_N2;
+  }
+  return run_adamw(params, gbar, m, v, d, hparams, step, n2_dev, stats_in ? max_norm : 0.0,
+                   params_bf16_out, stream);
 }
 
 int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs_dtype dtype,

@@ -37,6 +37,7 @@ struct StreamParams {
   float* p;    // fused AdamW only
   float* m;
   float* v;
+  uint16_t* p16; // fused AdamW, mixed precision: bf16 copy of the updated parameters, may be null
   double* chunk_out; // 4 doubles per chunk: n2, S, Q, 0
   AdamScalars adam;
 };
@@ -101,6 +102,24 @@ __device__ __forceinline__ void st_stream_32(float* p, const float4& lo, const f
   asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(lo.x),
                "f"(lo.y), "f"(lo.z), "f"(lo.w), "f"(hi.x), "f"(hi.y), "f"(hi.z), "f"(hi.w)
                : "memory");
+}
+
+// Two fp32 values rounded to nearest-even bf16, `lo` in the low half (the lower address).
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ uint16_t to_bf16(float x) {
+  return static_cast<uint16_t>(pack_bf16x2(x, 0.f) & 0xffffu);
+}
+// bf16 copy of four / eight consecutive parameters (8- / 16-byte aligned destination)
+__device__ __forceinline__ void st_bf16x4(uint16_t* dst, const float4& x) {
+  __stcs(reinterpret_cast<uint2*>(dst), make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w)));
+}
+__device__ __forceinline__ void st_bf16x8(uint16_t* dst, const float4& a, const float4& b) {
+  __stcs(reinterpret_cast<uint4*>(dst), make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w),
+                                                   pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w)));
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }

@@ -236,6 +236,10 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
           *reinterpret_cast<float4*>(st + OFF_P + tid * 16) = pw;
           *reinterpret_cast<float4*>(st + OFF_M + tid * 16) = pm;
           *reinterpret_cast<float4*>(st + OFF_V + tid * 16) = pv;
+          // the bf16 copy (mixed precision) goes straight from registers: 2 bytes per
+          // coordinate do not earn a stage segment
+          if (prm.p16)
+            st_bf16x4(prm.p16 + cg.lo + static_cast<int64_t>(i) * kBulkTile + tid * 4, pw);
         }
         if (prm.gbar)
           *reinterpret_cast<float4*>(st + OFF_GBAR + tid * 16) =

@@ -101,6 +101,7 @@ __device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t 
       prm.p[i] = w;
       prm.m[i] = m;
       prm.v[i] = v;
+      if (prm.p16) prm.p16[i] = to_bf16(w);
     }
   }
   sums[0] = row_n2;
@@ -140,6 +141,7 @@ __device__ __forceinline__ ChunkGeometry chunk_geometry(const StreamParams& prm,
     bits_f32 |= reinterpret_cast<uintptr_t>(prm.p) + static_cast<uintptr_t>(g.lo) * 4;
     bits_f32 |= reinterpret_cast<uintptr_t>(prm.m) + static_cast<uintptr_t>(g.lo) * 4;
     bits_f32 |= reinterpret_cast<uintptr_t>(prm.v) + static_cast<uintptr_t>(g.lo) * 4;
+    if (prm.p16) bits |= reinterpret_cast<uintptr_t>(prm.p16) + static_cast<uintptr_t>(g.lo) * 2;
   }
   g.aligned = ((bits | bits_f32) & 15) == 0;
   g.wide = (GT::kVec == 8) && (bits_f32 & 31) == 0;
@@ -222,6 +224,7 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
               st_stream_32(prm.p + base, pw[0], pw[NF4 - 1]);
               st_stream_32(prm.m + base, pm[0], pm[NF4 - 1]);
               st_stream_32(prm.v + base, pv[0], pv[NF4 - 1]);
+              if (prm.p16) st_bf16x8(prm.p16 + base, pw[0], pw[NF4 - 1]);
             }
           }
         } else {
@@ -231,6 +234,7 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
             st_stream_16(prm.p + base + 4 * q, pw[q]);
             st_stream_16(prm.m + base + 4 * q, pm[q]);
             st_stream_16(prm.v + base + 4 * q, pv[q]);
+            if (prm.p16) st_bf16x4(prm.p16 + base + 4 * q, pw[q]);
           }
         }
       }
@@ -357,6 +361,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
         st_stream_16(prm.p + base, pw);
         st_stream_16(prm.m + base, pm);
         st_stream_16(prm.v + base, pv);
+        if (prm.p16) st_bf16x4(prm.p16 + base, pw);
       }
     } else if (base < hi) {
       float sums[3];

@@ -228,7 +228,7 @@ template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
     adamw_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,
                  float* __restrict__ v, int64_t d, const AdamScalars a,
-                 const double* __restrict__ n2_dev, double max_norm) {
+                 const double* __restrict__ n2_dev, double max_norm, uint16_t* __restrict__ p16) {
   const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
   grid_dependency_wait();
   float scale = 1.f;
@@ -253,6 +253,7 @@ __global__ void __launch_bounds__(kThreads)
       st_stream_16(p + 4 * i, p0);
       st_stream_16(m + 4 * i, m0);
       st_stream_16(v + 4 * i, v0);
+      if (p16) st_bf16x4(p16 + 4 * i, p0);
       adamw_elem(a, scale * g1.x, p1.x, m1.x, v1.x);
       adamw_elem(a, scale * g1.y, p1.y, m1.y, v1.y);
       adamw_elem(a, scale * g1.z, p1.z, m1.z, v1.z);
@@ -260,6 +261,7 @@ __global__ void __launch_bounds__(kThreads)
       st_stream_16(p + 4 * j, p1);
       st_stream_16(m + 4 * j, m1);
       st_stream_16(v + 4 * j, v1);
+      if (p16) st_bf16x4(p16 + 4 * j, p1);
     }
     if (i < nvec) {
       const float4 gg = __ldcs(reinterpret_cast<const float4*>(g) + i);
@@ -271,6 +273,7 @@ __global__ void __launch_bounds__(kThreads)
       st_stream_16(p + 4 * i, pp);
       st_stream_16(m + 4 * i, mm);
       st_stream_16(v + 4 * i, vv);
+      if (p16) st_bf16x4(p16 + 4 * i, pp);
     }
     // tail (d % 4 elements) by the first threads of block 0
     const int64_t t = (nvec << 2) + threadIdx.x;
@@ -280,6 +283,7 @@ __global__ void __launch_bounds__(kThreads)
       p[t] = pp;
       m[t] = mm;
       v[t] = vv;
+      if (p16) p16[t] = to_bf16(pp);
     }
   } else {
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < d;
@@ -289,6 +293,7 @@ __global__ void __launch_bounds__(kThreads)
       p[i] = pp;
       m[i] = mm;
       v[i] = vv;
+      if (p16) p16[i] = to_bf16(pp);
     }
   }
 }

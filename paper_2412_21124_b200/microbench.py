@@ -7,8 +7,8 @@ Timing: CUDA events on the launching stream around `steps` back-to-back calls af
 `warmup` calls; calls shorter than ~50 us are captured in a CUDA graph and the replays are
 timed, so that the figure is device time and not the host's per-call cost.  Points whose working set is smaller than twice the L2 rotate over several
 independent buffer sets so that every call reads cold data.  GB/s counts algorithmic bytes:
-fused (K*s + 24) per coordinate (+4 with --gbar), normtest K*s + 4, adamw 28, persample 4
-per matrix element.
+fused (K*s + 24) per coordinate (+4 with --gbar, +2 with --mixed), normtest K*s + 4,
+adamw 28 (+2 with --mixed), persample 4 per matrix element.
 """
 import argparse
 import json
@@ -43,10 +43,14 @@ def bytes_per_call(call, d, K, esz, gbar, b):
 
 
 def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b=4096, dev="cuda",
-              graph=None):
+              graph=None, mixed=False):
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     esz = 2 if dtype == "bf16" else 4
     nbytes = bytes_per_call(call, d, K, esz, gbar, b)
+    if mixed:  # the bf16 copy of the parameters: 2 more bytes per coordinate
+        if call not in ("fused", "adamw"):
+            raise SystemExit("--mixed applies to the fused and adamw calls")
+        nbytes += 2 * d
     n_sets = 1 if nbytes >= 2 * L2_BYTES else -(-2 * L2_BYTES // nbytes) + 1
     offs = synth.equal_shard_offsets(d, n_shards) if n_shards > 1 else None
     sets = []
@@ -68,18 +72,26 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
             s["stats"] = B.alloc_persample_stats(b, d, dev)
             s["gbar"] = torch.zeros(d, dtype=torch.float32, device=dev)
         s["b_next"] = torch.zeros(1, dtype=torch.int64, device=dev)
-        if call == "fused":  # marshal once; each timed call is then a single C call
+        if mixed:
+            s["p16"] = torch.zeros(d, dtype=torch.bfloat16, device=dev)
+        if call == "fused" and not mixed:  # marshal once; each timed call is then a single C call
             s["prepared"] = B.FusedStep(s["grads"], s["stats"], s.get("gbar"), s["b_next"], s["p"],
                                         s["m"], s["v"], HP, shard_offsets=offs)
         sets.append(s)
 
     def one(i):
         s = sets[i % n_sets]
-        if call == "fused":
+        if call == "fused" and mixed:
+            B.abs_normtest_adamw_mixed(s["grads"], 0.1, 512, s["stats"], s.get("gbar"), s["b_next"],
+                                       s["p"], s["m"], s["v"], s["p16"], HP, 100 + i,
+                                       shard_offsets=offs)
+        elif call == "fused":
             s["prepared"].run(0.1, 512, 100 + i)
         elif call == "normtest":
             B.abs_norm_test(s["grads"], 0.1, 512, s["stats"], s["gbar"], s["b_next"],
                             shard_offsets=offs)
+        elif call == "adamw" and mixed:
+            B.abs_adamw_step_mixed(s["p"], s["gbar"], s["m"], s["v"], s["p16"], HP, 100 + i)
         elif call == "adamw":
             B.abs_adamw_step(s["p"], s["gbar"], s["m"], s["v"], HP, 100 + i)
         else:
@@ -129,7 +141,8 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
         torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     out = {"call": call, "d": d, "K": K, "dtype": dtype, "n_shards": n_shards, "gbar": bool(gbar),
-           "steps": steps, "buffer_sets": n_sets, "cuda_graph": bool(graph), "ms": ms,
+           "mixed": bool(mixed), "steps": steps, "buffer_sets": n_sets, "cuda_graph": bool(graph),
+           "ms": ms,
            "bytes": nbytes, "GBps": nbytes / (ms * 1e-3) / 1e9}
     if call == "persample":
         out["b"] = b
@@ -147,6 +160,8 @@ def main(argv=None):
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--gbar", action="store_true", help="fused: also write gbar")
+    ap.add_argument("--mixed", action="store_true",
+                    help="fused / adamw: also write the bf16 copy of the parameters")
     ap.add_argument("--sweep", action="store_true", help="fused call over the d x K x dtype grid")
     ap.add_argument("--graph", choices=["auto", "on", "off"], default="auto",
                     help="time replays of a captured CUDA graph (auto: for calls under 50 us)")
@@ -157,7 +172,8 @@ def main(argv=None):
     graph = {"auto": None, "on": True, "off": False}[args.graph]
     if not args.sweep:
         print(json.dumps(run_point(args.call, args.d, args.K, args.dtype, args.shards, args.steps,
-                                   args.warmup, args.gbar, args.b, graph=graph)), flush=True)
+                                   args.warmup, args.gbar, args.b, graph=graph,
+                                   mixed=args.mixed)), flush=True)
         return
     for dtype in ("bf16", "f32"):
         esz = 2 if dtype == "bf16" else 4

@@ -274,6 +274,26 @@ def test_clipped_adamw_rejects(L):
     assert f(FAKE, FAKE, FAKE, FAKE, 10, r, 0, 1.0, FAKE, None) == binding.ABS_ERR_RANGE
 
 
+def test_mixed_precision_rejects(L):
+    hp = binding.abs_adamw_hparams(1e-3, 0.9, 0.999, 1e-8, 0.1)
+    r = ctypes.byref(hp)
+    f = L.abs_adamw_step_mixed
+    assert f(FAKE, FAKE, FAKE, FAKE, None, 10, r, 1, 0.0, None, None) == binding.ABS_ERR_NULL
+    assert f(FAKE, FAKE, FAKE, FAKE, FAKE + 1, 10, r, 1, 0.0, None, None) == binding.ABS_ERR_ALIGN
+    assert f(None, FAKE, FAKE, FAKE, FAKE, 10, r, 1, 0.0, None, None) == binding.ABS_ERR_NULL
+    assert f(FAKE, FAKE, FAKE, FAKE, FAKE, 0, r, 1, 0.0, None, None) == binding.ABS_ERR_RANGE
+    # clipping is on exactly when stats_in is given: then max_norm must be finite and positive
+    assert f(FAKE, FAKE, FAKE, FAKE, FAKE, 10, r, 1, 0.0, FAKE, None) == binding.ABS_ERR_RANGE
+    assert f(FAKE, FAKE, FAKE, FAKE, FAKE, 10, r, 1, math.inf, FAKE, None) == binding.ABS_ERR_RANGE
+    assert f(FAKE, FAKE, FAKE, FAKE, FAKE, 10, r, 1, 1.0, FAKE + 4, None) == binding.ABS_ERR_ALIGN
+    base = _nt_args()[:-1]
+    g = L.abs_normtest_adamw_mixed
+    assert g(*(base + [FAKE, FAKE, FAKE, None, r, 1, None])) == binding.ABS_ERR_NULL
+    assert g(*(base + [FAKE, FAKE, FAKE, FAKE + 1, r, 1, None])) == binding.ABS_ERR_ALIGN
+    assert g(*(base + [None, FAKE, FAKE, FAKE, r, 1, None])) == binding.ABS_ERR_NULL
+    assert g(*(base + [FAKE, FAKE, FAKE, FAKE, r, 0, None])) == binding.ABS_ERR_RANGE
+
+
 def test_adamw_rejects_pointers(L):
     hp = _hp()
     r = ctypes.byref(hp)

@@ -476,6 +476,88 @@ def test_norm_test_then_clipped_adamw(max_norm, d, shift):
         assert torch.equal(q, views[0]) and torch.equal(mq, views[1]) and torch.equal(vq, views[2])
 
 
+# ------------------------------------------------------------------- mixed precision
+def bf16_bits(t):
+    return t.detach().cpu().view(torch.int16).numpy().view(np.uint16)
+
+
+def guarded_bf16(n, shift=0):
+    buf = torch.full((n + 2 * GUARD + shift,), 7.0, dtype=torch.bfloat16, device=DEV)
+    return buf, buf[GUARD + shift:GUARD + shift + n]
+
+
+def check_bf16_copy(p16_buf, p16, p_f32, n, shift):
+    """The bf16 copy is the stored fp32 value rounded to nearest even, bit for bit (the oracle
+    decides the code from the same fp32 value the kernel rounded), and nothing else was written."""
+    want = orc.bf16_round(to_host(p_f32))
+    assert np.array_equal(bf16_bits(p16), want)
+    assert bool((p16_buf[:GUARD + shift] == 7.0).all())
+    assert bool((p16_buf[GUARD + shift + n:] == 7.0).all())
+
+
+@pytest.mark.parametrize("K,dtype,d,offs,shift", [
+    (8, torch.bfloat16, 5 * 8192 + 777, None, 0),        # staged kernel + ragged last chunk
+    (8, torch.bfloat16, 3 * 8192, None, 1),              # copy off 16-byte alignment: scalar rows
+    (4, torch.float32, 50_001, [0, 5, 20_000, 50_001], 0),
+    (2, torch.bfloat16, 70_003, None, 0),                # 256-bit stores
+    (5, torch.bfloat16, 33_000, None, 0),
+    (32, torch.bfloat16, 20_481, None, 0),               # split kernel
+    (20, torch.float32, 9_999, None, 0),
+], ids=["k8", "k8-shifted", "k4-f32-shards", "k2", "k5", "k32", "k20-f32"])
+def test_mixed_precision_fused_step(K, dtype, d, offs, shift):
+    """abs_normtest_adamw_mixed = abs_normtest_adamw bit for bit, plus the bf16 copy."""
+    eta, b_cur, step = 0.1, 64, 5
+    grads, ref = make_case(K, d, dtype, eta, b_cur, seed=1600 + K, shard_offsets=offs)
+    n_sh = 1 if offs is None else len(offs) - 1
+    outs = []
+    for mixed in (False, True):
+        p, m, v = synth.adam_state(d, 1601, DEV, zero_moments=False)
+        stats = absnt.alloc_stats(d, n_sh, DEV)
+        gbar = torch.empty(d, dtype=torch.float32, device=DEV)
+        b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+        if mixed:
+            p16_buf, p16 = guarded_bf16(d, shift)
+            absnt.abs_normtest_adamw_mixed(grads, eta, b_cur, stats, gbar, b_next, p, m, v, p16, HP,
+                                           step, shard_offsets=offs)
+        else:
+            absnt.abs_normtest_adamw(grads, eta, b_cur, stats, gbar, b_next, p, m, v, HP, step,
+                                     shard_offsets=offs)
+        torch.cuda.synchronize()
+        outs.append((p, m, v, gbar, absnt.read_stats(stats, n_sh), int(b_next.item())))
+    for a, b in zip(outs[0][:4], outs[1][:4]):
+        assert torch.equal(a, b)
+    # an output off 16-byte alignment moves the rows to the element-wise path, whose partial sums
+    # group differently (same values, different fp32 row grouping)
+    rel = 0.0 if shift == 0 else 1e-7
+    for key in ("n2", "S"):
+        assert abs(outs[0][4][key] - outs[1][4][key]) <= rel * outs[0][4][key]
+    assert outs[0][5] == outs[1][5] == ref["b_next"]
+    check_bf16_copy(p16_buf, p16, outs[1][0], d, shift)
+    assert np.array_equal(bf16_bits(p16), bf16_bits(outs[1][0].to(torch.bfloat16)))
+
+
+@pytest.mark.parametrize("d,shift,clip", [(100_003, 0, False), (100_003, 1, False), (4096, 0, True),
+                                          (50_001, 3, True), (7, 0, False)])
+def test_mixed_precision_adamw_step(d, shift, clip):
+    grads, ref = make_case(4, d, torch.float32, 0.1, 64, seed=1650 + d % 5)
+    stats = absnt.alloc_stats(d, 1, DEV)
+    gbar = torch.empty(d, dtype=torch.float32, device=DEV)
+    b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+    absnt.abs_norm_test(grads, 0.1, 64, stats, gbar, b_next)
+    p, m, v = synth.adam_state(d, 1651, DEV, zero_moments=False)
+    q, mq, vq = p.clone(), m.clone(), v.clone()
+    p16_buf, p16 = guarded_bf16(d, shift)
+    if clip:
+        absnt.abs_adamw_step_clipped(q, gbar, mq, vq, HP, 3, 0.05, stats)
+        absnt.abs_adamw_step_mixed(p, gbar, m, v, p16, HP, 3, max_norm=0.05, stats_in=stats)
+    else:
+        absnt.abs_adamw_step(q, gbar, mq, vq, HP, 3)
+        absnt.abs_adamw_step_mixed(p, gbar, m, v, p16, HP, 3)
+    torch.cuda.synchronize()
+    assert torch.equal(p, q) and torch.equal(m, mq) and torch.equal(v, vq)
+    check_bf16_copy(p16_buf, p16, p, d, shift)
+
+
 # --------------------------------------------------------------------- per-sample form
 def persample_check(G, eta):
     b, d = G.shape

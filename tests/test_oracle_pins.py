@@ -453,6 +453,40 @@ def test_clipped_adamw_against_torch_clip_grad_norm():
 
 
 # ------------------------------------------------------------------- thread independence
+def test_bf16_round_against_torch_and_hand_cases():
+    """The bfloat16 working copy: against torch's conversion on random values and around every
+    kind of boundary, and against hand-worked ties (1 + 2^-8 is halfway between the bfloat16
+    neighbours 1 and 1 + 2^-7: ties go to the even significand)."""
+    rng = np.random.default_rng(77)
+    x = np.concatenate([
+        rng.standard_normal(20000).astype(np.float32),
+        (rng.standard_normal(2000) * 1e-30).astype(np.float32),
+        (rng.standard_normal(2000) * 1e30).astype(np.float32),
+        np.array([0.0, -0.0, 1.0, -1.0, np.inf, -np.inf, 3.3895314e38, -3.3895314e38,
+                  3.4028235e38, 1e-45, -1e-45, 1.17549435e-38, 9.18e-41], dtype=np.float32)])
+    # exact ties and their neighbours: k * 2^-8 + tiny offsets around odd k
+    base = (1.0 + np.arange(0, 64) * 2.0 ** -8).astype(np.float32)
+    ties = np.concatenate([base, np.nextafter(base, np.float32(2)), np.nextafter(base, np.float32(0)),
+                           -base])
+    x = np.concatenate([x, ties]).astype(np.float32)
+    got = orc.bf16_round(x)
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(got, want)
+    # hand-worked: 1 = 0x3F80; 1 + 2^-7 = 0x3F81; 1 + 2^-6 = 0x3F82
+    hand = {1.0 + 2.0 ** -8: 0x3F80,               # tie between 0x3F80 and 0x3F81 -> even
+            1.0 + 2.0 ** -7 + 2.0 ** -8: 0x3F82,   # tie between 0x3F81 and 0x3F82 -> even
+            1.0 + 2.0 ** -8 + 2.0 ** -20: 0x3F81,  # just above the tie
+            -(1.0 + 2.0 ** -8): 0xBF80,
+            0.5: 0x3F00, 3.0: 0x4040}
+    for val, code in hand.items():
+        assert int(orc.bf16_round(np.array([val], dtype=np.float32))[0]) == code, val
+    # the largest finite bfloat16 is 0x7F7F; halfway to 2^128 and beyond rounds to infinity
+    big = np.array([3.3895314e38, 3.3961775e38, 3.4028235e38], dtype=np.float32)
+    assert list(orc.bf16_round(big)) == [0x7F7F, 0x7F80, 0x7F80]
+    nan = orc.bf16_round(np.array([np.nan], dtype=np.float32))[0]
+    assert (nan & 0x7F80) == 0x7F80 and (nan & 0x007F) != 0
+
+
 def test_thread_count_does_not_change_results():
     code = (
         "import sys, numpy as np; sys.path.insert(0, %r)\n"
