@@ -309,8 +309,8 @@ class FusedStep:
     """
 
     def __init__(self, grads, stats_out, gbar_out, b_next_out, params, m, v, hparams,
-                 shard_offsets=None):
-        self._keep = (list(grads), stats_out, gbar_out, b_next_out, params, m, v)
+                 shard_offsets=None, params_bf16_out=None):
+        self._keep = (list(grads), stats_out, gbar_out, b_next_out, params, m, v, params_bf16_out)
         self._table, self._K, self._d, self._code = _grad_table(grads)
         self._offs, self._n_shards = _offsets(shard_offsets)
         for t, name in ((params, "params"), (m, "m"), (v, "v")):
@@ -322,12 +322,21 @@ class FusedStep:
         self._ptrs = (stats_out.data_ptr(), gbar_out.data_ptr() if gbar_out is not None else None,
                       b_next_out.data_ptr(), params.data_ptr(), m.data_ptr(), v.data_ptr())
         self._fn = lib().abs_normtest_adamw
+        self._p16 = None
+        if params_bf16_out is not None:  # mixed precision: also the bf16 copy of the parameters
+            _check_bf16_vec(params_bf16_out, self._d, "params_bf16_out")
+            self._p16 = params_bf16_out.data_ptr()
+            self._fn = lib().abs_normtest_adamw_mixed
 
     def run(self, eta, b_cur, step, stream=None):
         st, gb, bn, p, m, v = self._ptrs
-        rc = self._fn(self._table, self._K, self._d, self._code, self._offs, self._n_shards, eta,
-                      b_cur, st, gb, bn, p, m, v, self._hp_ref, step,
-                      torch.cuda.current_stream().cuda_stream if stream is None else _stream(stream))
+        cu_stream = torch.cuda.current_stream().cuda_stream if stream is None else _stream(stream)
+        if self._p16 is None:
+            rc = self._fn(self._table, self._K, self._d, self._code, self._offs, self._n_shards,
+                          eta, b_cur, st, gb, bn, p, m, v, self._hp_ref, step, cu_stream)
+        else:
+            rc = self._fn(self._table, self._K, self._d, self._code, self._offs, self._n_shards,
+                          eta, b_cur, st, gb, bn, p, m, v, self._p16, self._hp_ref, step, cu_stream)
         if rc != ABS_OK:
             raise AbsError(rc, "abs_normtest_adamw")
 

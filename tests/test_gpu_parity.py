@@ -285,6 +285,13 @@ def test_prepared_fused_step_matches_plain_call():
         outs.append((stats[:2].clone(), gbar, p, m, v, b_next))
     for a, b in zip(*outs):
         assert torch.equal(a, b)
+    # the prepared object with a bf16 copy of the parameters
+    p, m, v = synth.adam_state(d, 761, DEV, zero_moments=False)
+    p16 = torch.zeros(d, dtype=torch.bfloat16, device=DEV)
+    step = absnt.FusedStep(grads, stats, gbar, b_next, p, m, v, HP, params_bf16_out=p16)
+    step.run(0.1, 64, 4)
+    torch.cuda.synchronize()
+    assert torch.equal(p, outs[0][2]) and torch.equal(p16, p.to(torch.bfloat16))
 
 
 def test_calls_can_be_captured_in_a_cuda_graph():
