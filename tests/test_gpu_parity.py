@@ -607,6 +607,17 @@ def test_persample_shapes(b, d, ld, shift):
     persample_check(G, 0.1)
 
 
+def test_persample_more_rows_than_one_grid_dimension_of_512_row_blocks():
+    """b above 65535 x 512 rows: the row blocks must grow past 512 rows to fit the grid."""
+    b, d, ld = 65535 * 512 + 70_001, 3, 4
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(99)
+    buf = torch.empty(b * ld, dtype=torch.float32, device=DEV)
+    buf.normal_(generator=gen)
+    buf.mul_(0.3).add_(0.05)
+    persample_check(buf.view(b, ld)[:, :d], 0.1)
+
+
 def test_persample_matches_worker_form_factor():
     K, d = 8, 30_001
     grads, ref = make_case(K, d, torch.float32, 0.1, 1, seed=1300)
