@@ -47,7 +47,7 @@ typedef enum {
   ABS_ERR_TOO_LARGE = -7 /* the problem needs more built-in scratch than the library holds */
 } abs_status;
 
-enum { ABS_MAX_WORKERS = 32, ABS_MAX_SHARDS = 128 };
+enum { ABS_MAX_WORKERS = 64, ABS_MAX_SHARDS = 128 };
 
 /* AdamW hyper-parameters (alpha, beta1, beta2, epsilon, lambda of Algorithm 1). */
 typedef struct {

@@ -200,11 +200,11 @@ cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
 }
 
 // More than 16 workers: the split kernel, four coordinates per thread-row (bf16 gradients
-// are then read with 8-byte loads).
-template <typename GT, bool EXACT, bool ADAM>
+// are then read with 8-byte loads).  KB bounds the worker count of the instantiation.
+template <typename GT, bool EXACT, bool ADAM, int KB = 32>
 cudaError_t launch_split(const StreamParams& prm, cudaStream_t st) {
   using G4 = typename std::conditional<std::is_same<GT, BF16>::value, BF16H, GT>::type;
-  return launch_pdl(normtest_split_kernel<G4, 32, EXACT, ADAM, !ADAM>,
+  return launch_pdl(normtest_split_kernel<G4, KB, EXACT, ADAM, !ADAM>,
                     dim3(static_cast<unsigned>(prm.n_chunks)), dim3(kThreads), st, prm);
 }
 
@@ -221,7 +221,12 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
     case 8: return launch_one<GT, 8, true, ADAM>(prm, st);
     case 16: return launch_one<GT, 16, true, ADAM>(prm, st);
     case 32: return launch_split<GT, true, ADAM>(prm, st);
+    case 64:  // bf16: four unrolled groups of 16; fp32 spills in that form and takes the loop
+      if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, 64>(prm, st);
+      else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
     default:
+      // 33..64 workers (e.g. the J*M micro-batch gradients of one step): run-time groups of 8
+      if (K > 32) return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
       if (K < 8) return launch_one<GT, 8, false, ADAM>(prm, st);
       if (K < 16) return launch_one<GT, 16, false, ADAM>(prm, st);
       // 17..31 workers.  Measured at K=20/24: the run-time loop over groups of 8 wins for

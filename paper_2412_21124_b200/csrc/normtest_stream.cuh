@@ -20,6 +20,8 @@
 #pragma once
 #include <cooperative_groups.h>
 
+#include <type_traits>
+
 #include "abs_device.cuh"
 
 namespace absnt {
@@ -295,8 +297,10 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
                                                  double& acc_S, double& acc_Q) {
   constexpr int V = GT::kVec;
   static_assert(V == 4, "split path: four coordinates per thread-row");
-  // exact K: compile-time halves of 16; any other K: a run-time loop over groups of 8
-  constexpr int H = EXACT ? 16 : 8;
+  // exact K: compile-time groups of 16; any other K: a run-time loop over groups of 32 bytes
+  // per coordinate quad in registers (8 fp32 vectors, 16 bf16 vectors); full groups run
+  // without per-worker predicates, only the last, partial one tests k < K
+  constexpr int H = (EXACT || sizeof(typename GT::raw_t) <= 8) ? 16 : 8;
   static_assert(KB % H == 0, "groups");
   const int n_groups = EXACT ? KB / H : (K + H - 1) / H;
   const int tid = threadIdx.x;
@@ -319,19 +323,19 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
         pm = ld_state_16(prm.m + base);
         pv = ld_state_16(prm.v + base);
       }
-#pragma unroll(EXACT ? KB / H : 1)
-      for (int h = 0; h < n_groups; ++h) {
+      auto group = [&](int h, auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
         typename GT::raw_t raw[H];
 #pragma unroll
         for (int k = 0; k < H; ++k)
-          if (EXACT || h * H + k < K)
+          if (FULL || h * H + k < K)
             raw[k] = GT::load_vec(
                 reinterpret_cast<const typename GT::scalar*>(prm.grads[h * H + k]) + base);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
 #pragma unroll
           for (int k = 0; k < H; ++k)
-            if (EXACT || h * H + k < K) {
+            if (FULL || h * H + k < K) {
               const float g = GT::elem(raw[k], e);
               if (h == 0 && k == 0) c[e] = g;
               s[e] += static_cast<typename GT::sum_t>(g);
@@ -340,6 +344,11 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
               if (WITHQ) q[e] = fmaf(g, g, q[e]);
             }
         }
+      };
+#pragma unroll(EXACT ? KB / H : 1)
+      for (int h = 0; h < n_groups; ++h) {
+        if (EXACT || (h + 1) * H <= K) group(h, std::true_type{});
+        else group(h, std::false_type{});
       }
       float gb[V];
       float* w4 = reinterpret_cast<float*>(&pw);

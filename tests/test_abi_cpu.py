@@ -199,7 +199,7 @@ FAKE = 0x10000  # a non-null, 16-byte aligned value that is never dereferenced
 
 def _nt_args(**over):
     K = over.pop("K", 2)
-    table = over.pop("table", (ctypes.c_void_p * 32)(*([FAKE] * 32)))
+    table = over.pop("table", (ctypes.c_void_p * 64)(*([FAKE] * 64)))
     a = dict(grads=table, K=K, d=100, dtype=0, offs=None, n_shards=1, eta=0.1, b_cur=8,
              stats=FAKE, gbar=FAKE, b_next=FAKE, stream=None)
     a.update(over)
@@ -218,7 +218,7 @@ def _offs(*vals):
     (dict(b_next=None), binding.ABS_ERR_NULL),
     (dict(dtype=2), binding.ABS_ERR_DTYPE),
     (dict(K=0), binding.ABS_ERR_RANGE),
-    (dict(K=33), binding.ABS_ERR_RANGE),
+    (dict(K=65), binding.ABS_ERR_RANGE),
     (dict(d=0), binding.ABS_ERR_RANGE),
     (dict(b_cur=0), binding.ABS_ERR_RANGE),
     (dict(eta=0.0), binding.ABS_ERR_RANGE),
