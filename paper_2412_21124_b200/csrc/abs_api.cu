@@ -214,26 +214,37 @@ template <typename GT, bool ADAM>
 cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
   const int K = prm.K;
   switch (K) {
+    // every count up to 16 has an unrolled kernel of its own (a bucket kernel that predicates
+    // the absent workers runs 10-25% slower: bf16 K=12 5.6 vs 6.9 TB/s, fp32 K=6 5.5 vs 7.1)
     case 1: return launch_one<GT, 1, true, ADAM>(prm, st);
     case 2: return launch_one<GT, 2, true, ADAM>(prm, st);
     case 3: return launch_one<GT, 3, true, ADAM>(prm, st);
     case 4: return launch_one<GT, 4, true, ADAM>(prm, st);
+    case 5: return launch_one<GT, 5, true, ADAM>(prm, st);
+    case 6: return launch_one<GT, 6, true, ADAM>(prm, st);
+    case 7: return launch_one<GT, 7, true, ADAM>(prm, st);
     case 8: return launch_one<GT, 8, true, ADAM>(prm, st);
+    case 9: return launch_one<GT, 9, true, ADAM>(prm, st);
+    case 10: return launch_one<GT, 10, true, ADAM>(prm, st);
+    case 11: return launch_one<GT, 11, true, ADAM>(prm, st);
+    case 12: return launch_one<GT, 12, true, ADAM>(prm, st);
+    case 13: return launch_one<GT, 13, true, ADAM>(prm, st);
+    case 14: return launch_one<GT, 14, true, ADAM>(prm, st);
+    case 15: return launch_one<GT, 15, true, ADAM>(prm, st);
     case 16: return launch_one<GT, 16, true, ADAM>(prm, st);
     case 32: return launch_split<GT, true, ADAM>(prm, st);
     case 64:  // bf16: four unrolled groups of 16; fp32 spills in that form and takes the loop
       if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, 64>(prm, st);
       else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
+    case 24: return launch_split<GT, true, ADAM, 24>(prm, st);
+    case 48:
+      if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, 48>(prm, st);
+      else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
     default:
-      // 33..64 workers (e.g. the J*M micro-batch gradients of one step): run-time groups of 8
+      // 17..31 and 33..63 workers without a kernel of their own: run-time groups, the full
+      // groups unpredicated (bf16 K=20 5.3 TB/s, fp32 K=20 6.1, against 4.4 for a bucket kernel)
       if (K > 32) return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
-      if (K < 8) return launch_one<GT, 8, false, ADAM>(prm, st);
-      if (K < 16) return launch_one<GT, 16, false, ADAM>(prm, st);
-      // 17..31 workers.  Measured at K=20/24: the run-time loop over groups of 8 wins for
-      // fp32 gradients (5.27 vs 4.41 TB/s) and loses for bf16, whose 8-byte loads leave too
-      // few bytes in flight (4.20 vs 4.73 TB/s).
-      if constexpr (std::is_same<GT, F32>::value) return launch_split<GT, false, ADAM>(prm, st);
-      else return launch_one<GT, 32, false, ADAM>(prm, st);
+      return launch_split<GT, false, ADAM>(prm, st);
   }
 }
 

@@ -297,10 +297,11 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
                                                  double& acc_S, double& acc_Q) {
   constexpr int V = GT::kVec;
   static_assert(V == 4, "split path: four coordinates per thread-row");
-  // exact K: compile-time groups of 16; any other K: a run-time loop over groups of 32 bytes
+  // exact K: compile-time groups of 16 (of 8 when K is not a multiple of 16 and the vectors
+  // are 16 bytes); any other K: a run-time loop over groups of 32 bytes
   // per coordinate quad in registers (8 fp32 vectors, 16 bf16 vectors); full groups run
   // without per-worker predicates, only the last, partial one tests k < K
-  constexpr int H = (EXACT || sizeof(typename GT::raw_t) <= 8) ? 16 : 8;
+  constexpr int H = EXACT ? (KB % 16 == 0 ? 16 : 8) : (sizeof(typename GT::raw_t) <= 8 ? 16 : 8);
   static_assert(KB % H == 0, "groups");
   const int n_groups = EXACT ? KB / H : (K + H - 1) / H;
   const int tid = threadIdx.x;
