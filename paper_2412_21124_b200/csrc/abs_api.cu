@@ -176,13 +176,13 @@ cudaError_t launch_pdl_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
-// One (dtype, K bucket) instantiation: the bulk-async kernel where its stages leave room for
-// two or three CTAs per SM, else the register-direct kernel.
+// One (dtype, K) instantiation: the bulk-async kernel where its stages leave room for two or
+// three CTAs per SM, else the register-direct kernel.
 template <typename GT, int KB, bool EXACT, bool ADAM>
 cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
   const dim3 grid(static_cast<unsigned>(prm.n_chunks));
-  // Measured exceptions: the 512-coordinate tile loses to the register-direct kernel for the
-  // predicated K buckets (K=12: 5.46 vs 5.80 TB/s), and the unfused test -- 20 B per
+  // Measured exceptions: the 512-coordinate tile loses to the register-direct kernel when the
+  // worker loop is predicated (EXACT false; K=12: 5.46 vs 5.80 TB/s), and the unfused test -- 20 B per
   // coordinate at K=8 bf16, i.e. twice the coordinates per second -- is bound by instruction
   // issue, where the per-tile bookkeeping of the staged kernel costs 10% (5.95 vs 6.60 TB/s).
   constexpr BulkShape shape = bulk_shape<GT, KB, ADAM>();
@@ -214,8 +214,9 @@ template <typename GT, bool ADAM>
 cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
   const int K = prm.K;
   switch (K) {
-    // every count up to 16 has an unrolled kernel of its own (a bucket kernel that predicates
-    // the absent workers runs 10-25% slower: bf16 K=12 5.6 vs 6.9 TB/s, fp32 K=6 5.5 vs 7.1)
+    // every count up to 16 has an unrolled kernel of its own (one kernel for a range of counts,
+    // predicating the absent workers, ran 10-25% slower: bf16 K=12 5.6 vs 6.9 TB/s, fp32 K=6
+    // 5.5 vs 7.1)
     case 1: return launch_one<GT, 1, true, ADAM>(prm, st);
     case 2: return launch_one<GT, 2, true, ADAM>(prm, st);
     case 3: return launch_one<GT, 3, true, ADAM>(prm, st);
@@ -242,7 +243,8 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
       else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
     default:
       // 17..31 and 33..63 workers without a kernel of their own: run-time groups, the full
-      // groups unpredicated (bf16 K=20 5.3 TB/s, fp32 K=20 6.1, against 4.4 for a bucket kernel)
+      // groups unpredicated (bf16 K=20 5.3 TB/s, fp32 K=20 6.1, against 4.4 with every worker
+      // predicated)
       if (K > 32) return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
       return launch_split<GT, false, ADAM>(prm, st);
   }

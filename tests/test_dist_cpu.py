@@ -1,6 +1,7 @@
 """world_size-2 gloo test (CPU) of the multi-process host logic: index ranges cover the
 vector, per-rank sums combined in rank order reproduce the oracle's sharded totals and
-decision on every rank, and the timing reduction is a max."""
+decision on every rank, every rank's batch-size schedule advances identically, and the timing
+reduction is a max."""
 import os
 import socket
 import subprocess
@@ -26,9 +27,15 @@ out = adist.combine_rank_sums(mine["n2"], mine["S"], mine["Q"], K, eta, b_cur)
 offs = [adist.rank_range(d, r, world)[0] for r in range(world)] + [d]
 full = orc.norm_test(host, eta, b_cur, shard_offsets=offs, want_gbar=False)
 t = adist.max_over_ranks(1.0 + rank)
+# every rank advances its own copy of the schedule with the decision it computed
+from paper_2412_21124_b200 import binding
+sched = binding.abs_schedule_init(world, 2, 4, 4096, 8, 1)   # J = world, M = 2, microbatch 4: b = 16
+assert sched.b == b_cur and binding.abs_schedule_test_due(sched)
+binding.abs_schedule_advance(sched, out["b_next"])
 adist.barrier()
 print(json.dumps({"rank": rank, "out": out, "full": {k: full[k] for k in ("n2", "S", "Q", "T", "b_next", "flags")},
-                  "offs": offs, "tmax": t}))
+                  "offs": offs, "tmax": t,
+                  "sched": {k: getattr(sched, k) for k in ("J", "M", "micro", "b", "step", "samples")}}))
 """
 
 
@@ -72,3 +79,9 @@ def test_two_rank_combine_matches_oracle():
             assert r["out"][k] == r["full"][k], k  # rank-ordered sum == shard-ordered sum
         assert r["tmax"] == 2.0
     assert a["out"]["b_next"] > 16
+    # identical schedules on both ranks, the new batch a multiple of J*M that covers b_next
+    assert a["sched"] == b["sched"]
+    sc = a["sched"]
+    assert sc["b"] == sc["J"] * sc["M"] * sc["micro"] and sc["micro"] <= 8
+    assert sc["b"] >= min(a["out"]["b_next"], 4096) or sc["b"] == 4096 // (sc["J"] * sc["M"]) * sc["J"] * sc["M"]
+    assert sc["step"] == 2 and sc["samples"] == 16
