@@ -165,8 +165,65 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
   const int tid = threadIdx.x;
   const int64_t hi = cg.hi;
   const bool wide = cg.wide;
+  int64_t row_lo = cg.lo;
 
-  for (int64_t row_lo = cg.lo; row_lo < hi; row_lo += NT * V) {
+  // The test alone moves few bytes per coordinate (K*s + 4), so with few workers one thread-row
+  // of K vectors leaves too little in flight (K=4 bf16: 49 KB per SM, 68% DRAM utilisation,
+  // warps stalled on loads).  For K <= 4, while full aligned rows remain, 8/K of them are
+  // loaded before the first is consumed (eight vectors per thread, still three CTAs per SM);
+  // the rows are consumed in order, so the sums keep their shape.  Measured at d = 124M, bf16 /
+  // fp32: K=1 5.7 -> 6.4 / 5.1 -> 6.2 TB/s, K=2 5.9 -> 6.5 / 5.5 -> 6.5, K=4 5.9 -> 6.6 / 6.3 ->
+  // 6.5.  Sixteen vectors per thread at two CTAs per SM lose for bf16 (K=8: 6.6 -> 6.2).
+  constexpr int kRows = (!ADAM && EXACT && KB <= 4) ? 8 / KB : 1;
+  if constexpr (kRows > 1) {
+    while (cg.aligned && row_lo + static_cast<int64_t>(kRows) * NT * V <= hi) {
+      typename GT::raw_t rawr[kRows][KB];
+#pragma unroll
+      for (int r = 0; r < kRows; ++r)
+#pragma unroll
+        for (int k = 0; k < KB; ++k)
+          rawr[r][k] = GT::load_vec(reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) +
+                                    row_lo + static_cast<int64_t>(r) * NT * V +
+                                    static_cast<int64_t>(tid) * V);
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) {
+        const int64_t base = row_lo + static_cast<int64_t>(r) * NT * V + static_cast<int64_t>(tid) * V;
+        float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
+        float4 gbv[NF4];
+#pragma unroll
+        for (int q = 0; q < NF4; ++q) {
+          float gb[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float g[KB];
+#pragma unroll
+            for (int k = 0; k < KB; ++k) g[k] = GT::elem(rawr[r][k], 4 * q + j);
+            float dev2, sq;
+            const float mean = coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
+            gb[j] = mean;
+            row_n2 = fmaf(mean, mean, row_n2);
+            row_S += dev2;
+            row_Q += sq;
+          }
+          gbv[q] = make_float4(gb[0], gb[1], gb[2], gb[3]);
+        }
+        if (prm.gbar) {
+          if (V == 8 && wide) {
+            st_stream_32(prm.gbar + base, gbv[0], gbv[NF4 - 1]);
+          } else {
+#pragma unroll
+            for (int q = 0; q < NF4; ++q) st_stream_16(prm.gbar + base + 4 * q, gbv[q]);
+          }
+        }
+        acc_n2 += static_cast<double>(row_n2);
+        acc_S += static_cast<double>(row_S);
+        if (WITHQ) acc_Q += static_cast<double>(row_Q);
+      }
+      row_lo += static_cast<int64_t>(kRows) * NT * V;
+    }
+  }
+
+  for (; row_lo < hi; row_lo += NT * V) {
     const int64_t base = row_lo + static_cast<int64_t>(tid) * V;
     float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
 
