@@ -41,7 +41,11 @@ struct BulkShape {
 };
 template <typename GT, int KB, bool ADAM>
 __host__ __device__ constexpr BulkShape bulk_shape() {
-  if (2 * 3 * bulk_stage_bytes<GT, KB, ADAM>(1024) <= kSmemPerSM) return {1024, 3, 2};
+  if (2 * 3 * bulk_stage_bytes<GT, KB, ADAM>(1024) <= kSmemPerSM) {
+    // small stages (few workers): up to five of them, so that as many bytes stay in flight
+    const int fit = kSmemPerSM / (2 * bulk_stage_bytes<GT, KB, ADAM>(1024));
+    return {1024, fit > 5 ? 5 : fit, 2};
+  }
   if (3 * 3 * bulk_stage_bytes<GT, KB, ADAM>(512) <= kSmemPerSM) return {512, 3, 3};
   return {0, 0, 0};
 }
