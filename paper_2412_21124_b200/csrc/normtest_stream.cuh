@@ -356,11 +356,10 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
   static_assert(V == 4, "split path: four coordinates per thread-row");
   // exact K: compile-time groups of 16 (of 8 when K is not a multiple of 16 and the vectors
   // are 16 bytes); any other K: a run-time loop over groups of 32 bytes
-  // per coordinate quad in registers (8 fp32 vectors, 16 bf16 vectors); full groups run
-  // without per-worker predicates, only the last, partial one tests k < K
+  // per coordinate quad in registers (8 fp32 vectors, 16 bf16 vectors), then the remaining
+  // workers in unpredicated pieces of 8, 4, 2 and 1
   constexpr int H = EXACT ? (KB % 16 == 0 ? 16 : 8) : (sizeof(typename GT::raw_t) <= 8 ? 16 : 8);
   static_assert(KB % H == 0, "groups");
-  const int n_groups = EXACT ? KB / H : (K + H - 1) / H;
   const int tid = threadIdx.x;
   const int64_t hi = cg.hi;
 
@@ -381,32 +380,49 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
         pm = ld_state_16(prm.m + base);
         pv = ld_state_16(prm.v + base);
       }
-      auto group = [&](int h, auto full_tag) {
-        constexpr bool FULL = decltype(full_tag)::value;
-        typename GT::raw_t raw[H];
+      // N consecutive workers starting at k0, all present: loads first, then the arithmetic
+      auto group = [&](int k0, auto n_tag) {
+        constexpr int N = decltype(n_tag)::value;
+        typename GT::raw_t raw[N];
 #pragma unroll
-        for (int k = 0; k < H; ++k)
-          if (FULL || h * H + k < K)
-            raw[k] = GT::load_vec(
-                reinterpret_cast<const typename GT::scalar*>(prm.grads[h * H + k]) + base);
+        for (int k = 0; k < N; ++k)
+          raw[k] = GT::load_vec(
+              reinterpret_cast<const typename GT::scalar*>(prm.grads[k0 + k]) + base);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
 #pragma unroll
-          for (int k = 0; k < H; ++k)
-            if (FULL || h * H + k < K) {
-              const float g = GT::elem(raw[k], e);
-              if (h == 0 && k == 0) c[e] = g;
-              s[e] += static_cast<typename GT::sum_t>(g);
-              const float dv = g - c[e];
-              s2[e] = fmaf(dv, dv, s2[e]);
-              if (WITHQ) q[e] = fmaf(g, g, q[e]);
-            }
+          for (int k = 0; k < N; ++k) {
+            const float g = GT::elem(raw[k], e);
+            if (k0 == 0 && k == 0) c[e] = g;
+            s[e] += static_cast<typename GT::sum_t>(g);
+            const float dv = g - c[e];
+            s2[e] = fmaf(dv, dv, s2[e]);
+            if (WITHQ) q[e] = fmaf(g, g, q[e]);
+          }
         }
       };
-#pragma unroll(EXACT ? KB / H : 1)
-      for (int h = 0; h < n_groups; ++h) {
-        if (EXACT || (h + 1) * H <= K) group(h, std::true_type{});
-        else group(h, std::false_type{});
+      if constexpr (EXACT) {
+#pragma unroll
+        for (int h = 0; h < KB / H; ++h) group(h * H, std::integral_constant<int, H>{});
+      } else {
+        // whole groups in a run-time loop, then the remainder in pieces of 8, 4, 2, 1 workers:
+        // no load is predicated on the worker count
+        int k0 = 0;
+#pragma unroll 1
+        for (; k0 + H <= K; k0 += H) group(k0, std::integral_constant<int, H>{});
+        if (H > 8 && ((K - k0) & 8)) {
+          group(k0, std::integral_constant<int, 8>{});
+          k0 += 8;
+        }
+        if ((K - k0) & 4) {
+          group(k0, std::integral_constant<int, 4>{});
+          k0 += 4;
+        }
+        if ((K - k0) & 2) {
+          group(k0, std::integral_constant<int, 2>{});
+          k0 += 2;
+        }
+        if ((K - k0) & 1) group(k0, std::integral_constant<int, 1>{});
       }
       float gb[V];
       float* w4 = reinterpret_cast<float*>(&pw);
