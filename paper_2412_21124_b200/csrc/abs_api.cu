@@ -6,6 +6,7 @@
 #include <cstring>
 #include <mutex>
 #include <type_traits>
+#include <unordered_map>
 #include <utility>
 
 #include "abs_device.cuh"
@@ -155,13 +156,33 @@ int make_layout(int64_t d, const int64_t* shard_offsets, int n_shards, bool fuse
   return ABS_OK;
 }
 
+// Raises a kernel's dynamic shared-memory limit once per (kernel, device): the attribute call
+// costs about a microsecond of host time, which a launch-bound small-d loop would pay per step.
+cudaError_t allow_dynamic_smem(const void* kernel, size_t smem) {
+  static std::mutex mu;
+  static std::unordered_map<const void*, uint64_t> done;  // kernel -> bit per device
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const uint64_t bit = dev < 64 ? (uint64_t{1} << dev) : 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = done.find(kernel);
+    if (bit && it != done.end() && (it->second & bit)) return cudaSuccess;
+  }
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  done[kernel] |= bit;
+  return cudaSuccess;
+}
+
 // Launch with dynamic shared memory above the 48 KB default.
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                             cudaStream_t st, Args&&... args) {
-  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel),
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
+  cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(kernel), smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
