@@ -215,6 +215,34 @@ def test_more_than_32_workers(K, dtype):
                   grad_shift=1 if K == 48 else 0)
 
 
+def _random_case(i):
+    rng = np.random.default_rng(9000 + i)
+    K = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 11, 13, 16, 17, 23, 24, 31, 32, 33, 47, 48, 63, 64]))
+    d = int(rng.choice([1, 17, 255, 4096, 4097, 9_999, 40_000, 100_003, 262_144, 1_000_003]))
+    if K > 16:
+        d = min(d, 100_003)
+    dtype = torch.bfloat16 if rng.integers(2) else torch.float32
+    fused = bool(rng.integers(2))
+    n_sh = int(rng.choice([1, 1, 2, 5, 17]))
+    offs = None
+    if n_sh > 1 and d >= n_sh:
+        cuts = sorted(int(c) for c in rng.integers(0, d + 1, size=n_sh - 1))
+        offs = [0] + cuts + [d]
+    grad_shift = int(rng.choice([0, 0, 0, 1, 3]))
+    state_shift = int(rng.choice([0, 0, 1]))
+    return K, d, dtype, fused, offs, grad_shift, state_shift
+
+
+@pytest.mark.parametrize("i", range(40))
+def test_randomized_configurations(i):
+    """Seeded random draws over worker count, length, dtype, entry point, ragged shard cuts
+    (empty shards included) and buffer alignment: every combination goes through the same
+    element-by-element comparison with the oracle."""
+    K, d, dtype, fused, offs, grad_shift, state_shift = _random_case(i)
+    run_and_check(K, d, dtype, fused=fused, seed=9100 + i, shard_offsets=offs, grad_shift=grad_shift,
+                  state_shift=state_shift, zero_moments=bool(i % 2), step=1 + (i % 7))
+
+
 def test_fused_without_gbar_output():
     run_and_check(8, 40_000, torch.bfloat16, fused=True, seed=600, want_gbar=False)
 
