@@ -14,7 +14,8 @@
  *   - "device" pointers are memory of the CUDA device that is current on the calling
  *     thread; "host" pointers are ordinary memory read during the call only.
  *   - The caller owns every buffer.  The library allocates no device memory and
- *     keeps no state between calls (abs_last_cuda_error aside).
+ *     keeps no state between calls that a result depends on (what it does keep, on the
+ *     host: abs_last_cuda_error, and which kernel attributes it has set on which device).
  *   - Work is enqueued on `stream` (a cudaStream_t; NULL = the legacy default
  *     stream).  No call synchronises with the host; results are valid in stream order.
  *   - Return value: ABS_OK, or a negative abs_status.  On a negative status nothing
