@@ -258,16 +258,28 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
     case 64:  // bf16: four unrolled groups of 16; fp32 spills in that form and takes the loop
       if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, 64>(prm, st);
       else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
+    case 17: return launch_split<GT, true, ADAM, 17>(prm, st);
+    case 18: return launch_split<GT, true, ADAM, 18>(prm, st);
+    case 19: return launch_split<GT, true, ADAM, 19>(prm, st);
+    case 20: return launch_split<GT, true, ADAM, 20>(prm, st);
+    case 21: return launch_split<GT, true, ADAM, 21>(prm, st);
+    case 22: return launch_split<GT, true, ADAM, 22>(prm, st);
+    case 23: return launch_split<GT, true, ADAM, 23>(prm, st);
     case 24: return launch_split<GT, true, ADAM, 24>(prm, st);
+    case 25: return launch_split<GT, true, ADAM, 25>(prm, st);
+    case 26: return launch_split<GT, true, ADAM, 26>(prm, st);
+    case 27: return launch_split<GT, true, ADAM, 27>(prm, st);
+    case 28: return launch_split<GT, true, ADAM, 28>(prm, st);
+    case 29: return launch_split<GT, true, ADAM, 29>(prm, st);
+    case 30: return launch_split<GT, true, ADAM, 30>(prm, st);
+    case 31: return launch_split<GT, true, ADAM, 31>(prm, st);
     case 48:
       if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, 48>(prm, st);
       else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
     default:
-      // 17..31 and 33..63 workers without a kernel of their own: run-time groups, the full
-      // groups unpredicated (bf16 K=20 5.3 TB/s, fp32 K=20 6.1, against 4.4 with every worker
-      // predicated)
-      if (K > 32) return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
-      return launch_split<GT, false, ADAM>(prm, st);
+      // 33..63 workers without a kernel of their own: run-time groups and unpredicated pieces
+      // (5.6-6.1 TB/s; a kernel with compile-time groups runs at 6.4-6.7, as K = 17..32 show)
+      return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
   }
 }
 

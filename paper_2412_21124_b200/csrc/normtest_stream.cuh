@@ -354,12 +354,12 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
                                                  double& acc_S, double& acc_Q) {
   constexpr int V = GT::kVec;
   static_assert(V == 4, "split path: four coordinates per thread-row");
-  // exact K: compile-time groups of 16 (of 8 when K is not a multiple of 16 and the vectors
-  // are 16 bytes); any other K: a run-time loop over groups of 32 bytes
+  // exact K: compile-time groups of 16 and one group of K mod 16; any other K: a run-time loop
+  // over groups of 32 bytes
   // per coordinate quad in registers (8 fp32 vectors, 16 bf16 vectors), then the remaining
   // workers in unpredicated pieces of 8, 4, 2 and 1
-  constexpr int H = EXACT ? (KB % 16 == 0 ? 16 : 8) : (sizeof(typename GT::raw_t) <= 8 ? 16 : 8);
-  static_assert(KB % H == 0, "groups");
+  constexpr int H = EXACT ? 16 : (sizeof(typename GT::raw_t) <= 8 ? 16 : 8);
+  static_assert(EXACT || KB % H == 0, "groups");
   const int tid = threadIdx.x;
   const int64_t hi = cg.hi;
 
@@ -404,6 +404,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
       if constexpr (EXACT) {
 #pragma unroll
         for (int h = 0; h < KB / H; ++h) group(h * H, std::integral_constant<int, H>{});
+        if constexpr (KB % H != 0) group(KB / H * H, std::integral_constant<int, KB % H>{});
       } else {
         // whole groups in a run-time loop, then the remainder in pieces of 8, 4, 2, 1 workers:
         // no load is predicated on the worker count
