@@ -9,6 +9,10 @@ cross the wire.  This module holds that small host-side logic:
   combine_rank_sums   all-gather of {n2, S, Q} per rank, added in rank order on every
                       rank (so all ranks take the same bit-identical decision), then the
                       library's host-side decision
+  sharded_normtest_adamw
+                      the fused step on this rank's index range followed by that exchange:
+                      the multi-GPU form of FSDP-Norm (Sec. 3.3; Algorithm 1 with the shard
+                      sums "concatenated")
   max_over_ranks      max-reduction used for timing
 """
 import os
@@ -60,6 +64,44 @@ def combine_rank_sums(n2, S, Q, K, eta, b_cur, device="cpu", group=None):
         for j in range(3):
             tot[j] += vals[j]
     b_next, T, flags = binding.abs_decide(tot[1], tot[0], K, eta, b_cur)
+    return {"n2": tot[0], "S": tot[1], "Q": tot[2], "T": T, "flags": flags, "b_next": b_next}
+
+
+def _gather_rank_rows(local, group=None):
+    """all-gather of one small fp64 row per rank -> list of rows in rank order.  The row
+    travels on the device the backend works with (NCCL: this rank's GPU, gloo: the host)."""
+    if not (dist.is_initialized() and dist.get_world_size(group) > 1):
+        return [local.tolist()]
+    on_gpu = dist.get_backend(group) == "nccl"
+    if on_gpu and not local.is_cuda:
+        local = local.cuda()
+    if not on_gpu and local.is_cuda:
+        local = local.cpu()  # synchronises with the stream that wrote the sums
+    parts = [torch.empty_like(local) for _ in range(dist.get_world_size(group))]
+    dist.all_gather(parts, local.contiguous(), group=group)
+    return [part.tolist() for part in parts]
+
+
+def sharded_normtest_adamw(grads_local, eta, b_cur, stats_out, gbar_out, b_next_out, params_local,
+                           m_local, v_local, hparams, step, group=None):
+    """FSDP-Norm step (Sec. 3.3) with one process per GPU.  Every rank holds the same index
+    range [lo, hi) of all K gradient buffers and of params / m / v (`rank_range`) and passes
+    those slices.  The rank's GPU runs the fused norm-test + AdamW call on its range; the only
+    exchange is an all-gather of the three sums of the rank (24 bytes), added in rank order on
+    every rank, so that all ranks compute the same T and b_next bit for bit.  AdamW is
+    element-wise and needs no exchange.
+
+    `b_next_out` receives the local range's own decision (what the kernel wrote); the global
+    one is in the returned dict: n2, S, Q (NaN: the fused call does not compute it), T, flags,
+    b_next.  Synchronises the host with the stream (the sums are read back)."""
+    binding.abs_normtest_adamw(grads_local, eta, b_cur, stats_out, gbar_out, b_next_out,
+                               params_local, m_local, v_local, hparams, step)
+    local = stats_out.view(torch.float64)[binding.ABS_STAT_N2:binding.ABS_STAT_Q + 1]
+    tot = [0.0, 0.0, 0.0]
+    for row in _gather_rank_rows(local, group):  # rank order
+        for j in range(3):
+            tot[j] += row[j]
+    b_next, T, flags = binding.abs_decide(tot[1], tot[0], len(grads_local), eta, b_cur)
     return {"n2": tot[0], "S": tot[1], "Q": tot[2], "T": T, "flags": flags, "b_next": b_next}
 
 
