@@ -276,6 +276,18 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
     case 48:
       if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, 48>(prm, st);
       else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
+#define ABS_SPLIT_BF16_CASE(N)                                                              \
+  case N:                                                                                   \
+    if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, N>(prm, st); \
+    else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
+    // the multiples of four above 32 (J workers x M accumulation steps is one in practice)
+    ABS_SPLIT_BF16_CASE(36)
+    ABS_SPLIT_BF16_CASE(40)
+    ABS_SPLIT_BF16_CASE(44)
+    ABS_SPLIT_BF16_CASE(52)
+    ABS_SPLIT_BF16_CASE(56)
+    ABS_SPLIT_BF16_CASE(60)
+#undef ABS_SPLIT_BF16_CASE
     default:
       // 33..63 workers without a kernel of their own: run-time groups and unpredicated pieces
       // (5.6-6.1 TB/s; a kernel with compile-time groups runs at 6.4-6.7, as K = 17..32 show)

@@ -206,10 +206,13 @@ def test_many_workers_ragged_and_misaligned(K, dtype):
 
 
 @pytest.mark.parametrize("K,dtype", [(33, torch.bfloat16), (48, torch.float32), (64, torch.bfloat16),
-                                     (64, torch.float32)],
-                         ids=["k33-bf16", "k48-f32", "k64-bf16", "k64-f32"])
+                                     (64, torch.float32)]
+                         + [(K, torch.bfloat16) for K in (36, 40, 44, 48, 52, 56, 60)]
+                         + [(40, torch.float32), (47, torch.bfloat16)],
+                         ids=lambda x: str(x).replace("torch.", ""))
 def test_more_than_32_workers(K, dtype):
-    """33..64 buffers (e.g. the J*M micro-batch gradients of a step): run-time groups of 8."""
+    """33..64 buffers (e.g. the J*M micro-batch gradients of a step): compile-time groups for
+    bf16 multiples of four, run-time groups of 8 otherwise."""
     run_and_check(K, 2 * 4096 + 1_234, dtype, fused=True, seed=560 + K, zero_moments=False, step=3)
     run_and_check(K, 9_999, dtype, fused=False, seed=561 + K, shard_offsets=[0, 5, 4101, 9_999],
                   grad_shift=1 if K == 48 else 0)
