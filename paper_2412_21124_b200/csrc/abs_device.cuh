@@ -145,6 +145,24 @@ __device__ __forceinline__ void adamw_elem(const AdamScalars& a, float g, float&
   w = fmaf(a.decay, w, -((a.step_size * m) * inv));
 }
 
+// The same update for two adjacent coordinates with the packed fp32 instructions of sm_100
+// (fma/add/mul.f32x2: one issue slot for both lanes, each lane rounded exactly like the
+// scalar instruction, so the results are bit-identical to two adamw_elem calls).
+__device__ __forceinline__ void adamw_pair(const AdamScalars& a, float2 g, float2& w, float2& m,
+                                           float2& v) {
+  const float2 b1 = make_float2(a.beta1, a.beta1), b2 = make_float2(a.beta2, a.beta2);
+  m = __ffma2_rn(b1, m, __fmul2_rn(make_float2(a.omb1, a.omb1), g));
+  v = __ffma2_rn(b2, v, __fmul2_rn(__fmul2_rn(make_float2(a.omb2, a.omb2), g), g));
+  const float2 vh = __fmul2_rn(v, make_float2(a.inv_bc2, a.inv_bc2));
+  float2 root, inv;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root.x) : "f"(vh.x));
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root.y) : "f"(vh.y));
+  const float2 den = __fadd2_rn(root, make_float2(a.eps, a.eps));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv.x) : "f"(den.x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv.y) : "f"(den.y));
+  const float2 upd = __fmul2_rn(__fmul2_rn(make_float2(a.step_size, a.step_size), m), inv);
+  w = __ffma2_rn(make_float2(a.decay, a.decay), w, make_float2(-upd.x, -upd.y));
+}
 // Mean of K fp32 partial sums: s/K.  For K a power of two the product with 1/K is exact;
 // otherwise one residual correction makes K identical inputs return exactly that input.
 template <bool POW2>
@@ -154,6 +172,13 @@ __device__ __forceinline__ float mean_of_sum(float s, float inv_K, float neg_K) 
   return q;
 }
 
+template <bool POW2>
+__device__ __forceinline__ float2 mean_of_sum2(float2 s, float inv_K, float neg_K) {
+  const float2 ik = make_float2(inv_K, inv_K);
+  float2 q = __fmul2_rn(s, ik);
+  if (!POW2) q = __ffma2_rn(__ffma2_rn(make_float2(neg_K, neg_K), q, s), ik, q);
+  return q;
+}
 // Element types of the gradient buffers.
 struct F32 {
   static constexpr int kVec = 4; // elements per 16 bytes
@@ -167,6 +192,11 @@ struct F32 {
   }
   static __device__ __forceinline__ float elem(const uint4& r, int e) {
     return __uint_as_float(e == 0 ? r.x : e == 1 ? r.y : e == 2 ? r.z : r.w);
+  }
+  // coordinates 2*pi, 2*pi+1 of the vector
+  static __device__ __forceinline__ float2 pair(const uint4& r, int pi) {
+    return pi == 0 ? make_float2(__uint_as_float(r.x), __uint_as_float(r.y))
+                   : make_float2(__uint_as_float(r.z), __uint_as_float(r.w));
   }
   static __device__ __forceinline__ float load1(const void* base, int64_t i) {
     return __ldg(reinterpret_cast<const float*>(base) + i);
@@ -185,6 +215,10 @@ struct BF16 {
   static __device__ __forceinline__ float elem(const uint4& r, int e) {
     const uint32_t w = (e >> 1) == 0 ? r.x : (e >> 1) == 1 ? r.y : (e >> 1) == 2 ? r.z : r.w;
     return (e & 1) ? bf16_hi(w) : bf16_lo(w);
+  }
+  static __device__ __forceinline__ float2 pair(const uint4& r, int pi) {
+    const uint32_t w = pi == 0 ? r.x : pi == 1 ? r.y : pi == 2 ? r.z : r.w;
+    return make_float2(bf16_lo(w), bf16_hi(w));
   }
   static __device__ __forceinline__ float load1(const void* base, int64_t i) {
     return __uint_as_float(
@@ -210,6 +244,10 @@ struct BF16H {
   static __device__ __forceinline__ float elem(const uint2& r, int e) {
     const uint32_t w = (e >> 1) ? r.y : r.x;
     return (e & 1) ? bf16_hi(w) : bf16_lo(w);
+  }
+  static __device__ __forceinline__ float2 pair(const uint2& r, int pi) {
+    const uint32_t w = pi ? r.y : r.x;
+    return make_float2(bf16_lo(w), bf16_hi(w));
   }
   static __device__ __forceinline__ float load1(const void* base, int64_t i) {
     return BF16::load1(base, i);

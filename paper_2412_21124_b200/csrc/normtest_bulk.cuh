@@ -118,6 +118,10 @@ struct BulkGrad<BF16> {
     const uint32_t w = (j >> 1) ? r.y : r.x;
     return (j & 1) ? bf16_hi(w) : bf16_lo(w);
   }
+  __device__ __forceinline__ float2 pair(int jp) const {  // coordinates 2jp, 2jp+1
+    const uint32_t w = jp ? r.y : r.x;
+    return make_float2(bf16_lo(w), bf16_hi(w));
+  }
 };
 template <>
 struct BulkGrad<F32> {
@@ -127,6 +131,9 @@ struct BulkGrad<F32> {
   }
   __device__ __forceinline__ float elem(int j) const {
     return j == 0 ? r.x : j == 1 ? r.y : j == 2 ? r.z : r.w;
+  }
+  __device__ __forceinline__ float2 pair(int jp) const {
+    return jp ? make_float2(r.z, r.w) : make_float2(r.x, r.y);
   }
 };
 
@@ -214,23 +221,30 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
           pm = *reinterpret_cast<const float4*>(st + OFF_M + tid * 16);
           pv = *reinterpret_cast<const float4*>(st + OFF_V + tid * 16);
         }
-        float* w4 = reinterpret_cast<float*>(&pw);
-        float* m4 = reinterpret_cast<float*>(&pm);
-        float* v4 = reinterpret_cast<float*>(&pv);
+        float2* w2 = reinterpret_cast<float2*>(&pw);
+        float2* m2 = reinterpret_cast<float2*>(&pm);
+        float2* v2 = reinterpret_cast<float2*>(&pv);
         float gb[4];
         float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
+        // two coordinates per packed instruction; the row sums take the coordinates in
+        // index order, as the register-direct path does
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          float g[KB];
+        for (int jp = 0; jp < 2; ++jp) {
+          float2 g[KB];
 #pragma unroll
-          for (int k = 0; k < KB; ++k) g[k] = (EXACT || k < K) ? raw[k].elem(j) : 0.f;
-          float dev2, sq;
-          const float mean = coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
-          gb[j] = mean;
-          row_n2 = fmaf(mean, mean, row_n2);
-          row_S += dev2;
-          row_Q += sq;
-          if (ADAM) adamw_elem(prm.adam, mean, w4[j], m4[j], v4[j]);
+          for (int k = 0; k < KB; ++k)
+            g[k] = (EXACT || k < K) ? raw[k].pair(jp) : make_float2(0.f, 0.f);
+          float2 dev2, sq;
+          const float2 mean = coord_math_pair<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
+          gb[2 * jp] = mean.x;
+          gb[2 * jp + 1] = mean.y;
+          row_n2 = fmaf(mean.x, mean.x, row_n2);
+          row_n2 = fmaf(mean.y, mean.y, row_n2);
+          row_S += dev2.x;
+          row_S += dev2.y;
+          row_Q += sq.x;
+          row_Q += sq.y;
+          if (ADAM) adamw_pair(prm.adam, mean, w2[jp], m2[jp], v2[jp]);
         }
         acc_n2 += static_cast<double>(row_n2);
         acc_S += static_cast<double>(row_S);
