@@ -16,7 +16,10 @@
 // over more than 13 binades (8-bit significands in a 24-bit accumulator), and fp64
 // conversions would cost ~3% of bandwidth at the power cap.  Deviations g_k - gbar and
 // their squares (and, in the unfused kernel, g_k^2) are fp32 over at most V*K terms per
-// thread-row, then accumulated in fp64.
+// thread-row, then accumulated in fp64.  The fused kernels and the many-worker kernel do
+// this arithmetic two adjacent coordinates at a time with the packed fp32 instructions of
+// sm_100 (coord_math_pair, adamw_pair); every lane rounds like the scalar instruction, so
+// packed and scalar code give the same bits.
 #pragma once
 #include <cooperative_groups.h>
 
