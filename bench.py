@@ -16,6 +16,7 @@ import argparse
 import hashlib
 import json
 import os
+import re
 import statistics
 import sys
 import threading
@@ -53,12 +54,20 @@ def measured_peak():
 
 
 def kernel_source_hash():
+    """Hash of the kernel sources as the compiler sees them: comments, blank lines and
+    indentation do not count (no string literal in those files contains a comment marker)."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2412_21124_b200", "csrc")
     for name in sorted(os.listdir(csrc)):
-        with open(os.path.join(csrc, name), "rb") as f:
-            h.update(name.encode())
-            h.update(f.read())
+        with open(os.path.join(csrc, name), "r", encoding="utf-8") as f:
+            text = f.read()
+        text = re.sub(r"/\*.*?\*/", " ", text, flags=re.S)
+        h.update(name.encode())
+        for line in text.splitlines():
+            code = " ".join(line.split("//", 1)[0].split())
+            if code:
+                h.update(code.encode())
+                h.update(b"\n")
     return h.hexdigest()[:16]
 
 
