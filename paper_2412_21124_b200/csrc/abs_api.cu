@@ -202,12 +202,17 @@ cudaError_t launch_pdl_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
 template <typename GT, int KB, bool EXACT, bool ADAM>
 cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
   const dim3 grid(static_cast<unsigned>(prm.n_chunks));
-  // Measured exceptions: the 512-coordinate tile loses to the register-direct kernel when the
-  // worker loop is predicated (EXACT false; K=12: 5.46 vs 5.80 TB/s), and the unfused test -- 20 B per
-  // coordinate at K=8 bf16, i.e. twice the coordinates per second -- is bound by instruction
-  // issue, where the per-tile bookkeeping of the staged kernel costs 10% (5.95 vs 6.60 TB/s).
+  // Measured exceptions.  Fused: the 512-coordinate tile loses to the register-direct kernel
+  // when the worker loop is predicated (EXACT false; K=12: 5.46 vs 5.80 TB/s).  Unfused test
+  // (K*s + 4 bytes per coordinate, so more coordinates per second and more instructions per
+  // byte): staging wins by 1-9% for most worker counts (fp32 K=5 6.39 -> 6.96 TB/s, bf16 K=9
+  // 6.42 -> 6.87) but loses where the register-direct kernel is at its best: one or two
+  // workers (bf16 K=1 -37%, K=2 -7%; fp32 K=2 equal) and bf16 K=6 (-0.4%), K=8 (-2.8%).
   constexpr BulkShape shape = bulk_shape<GT, KB, ADAM>();
-  constexpr int tile = (!ADAM || (shape.tile == 512 && !EXACT)) ? 0 : shape.tile;
+  constexpr bool kBf16 = std::is_same<GT, BF16>::value;
+  constexpr bool staged_test = EXACT && KB >= 3 && !(kBf16 && (KB == 6 || KB == 8));
+  constexpr int tile = ADAM ? ((shape.tile == 512 && !EXACT) ? 0 : shape.tile)
+                            : (staged_test ? shape.tile : 0);
   if constexpr (tile > 0) {
     constexpr size_t smem =
         static_cast<size_t>(shape.stages) * bulk_stage_bytes<GT, KB, ADAM>(tile);
