@@ -18,8 +18,19 @@
  *     host: abs_last_cuda_error, and which kernel attributes it has set on which device).
  *   - Work is enqueued on `stream` (a cudaStream_t; NULL = the legacy default
  *     stream).  No call synchronises with the host; results are valid in stream order.
- *   - Return value: ABS_OK, or a negative abs_status.  On a negative status nothing
- *     was launched and no output was written.
+ *   - Return value: ABS_OK, or a negative abs_status.  Every status other than
+ *     ABS_ERR_CUDA comes from a check made before anything is launched: no output was
+ *     written.  ABS_ERR_CUDA reports a CUDA runtime call that failed.  A call enqueues one to
+ *     three kernels; if the failing call was a launch after the first, the earlier kernels
+ *     of the call may still run: the fused calls may then have updated params, m and v (and
+ *     gbar_out) in place while stats_out and b_next_out were not written, and repeating the
+ *     call would apply the update twice.  The refusal that can be foreseen is ruled out:
+ *     whether the device can co-schedule the thread-block cluster of the final reduction is
+ *     asked once per device before the first launch, and a single block is used if not.
+ *     What remains is a launch refused because the context is already broken.
+ *   - Aliasing: params, m and v are updated in place.  Apart from that, no output range may
+ *     share a byte with a gradient buffer or with another output of the same call; the
+ *     norm-test calls check this on the host and return ABS_ERR_ALIAS.
  *   - Results are deterministic: the same inputs give bit-identical outputs on every
  *     call, independent of how the hardware schedules thread blocks.
  */
@@ -45,7 +56,8 @@ typedef enum {
   ABS_ERR_ALIGN = -4,  /* a buffer is not aligned to its element size                  */
   ABS_ERR_DTYPE = -5,  /* dtype is not an abs_dtype                                    */
   ABS_ERR_CUDA = -6,   /* a CUDA call failed; see abs_last_cuda_error()                */
-  ABS_ERR_TOO_LARGE = -7 /* the problem needs more built-in scratch than the library holds */
+  ABS_ERR_TOO_LARGE = -7, /* the problem needs more built-in scratch than the library holds */
+  ABS_ERR_ALIAS = -8   /* an output overlaps a gradient buffer or another output        */
 } abs_status;
 
 enum { ABS_MAX_WORKERS = 64, ABS_MAX_SHARDS = 128 };
@@ -111,7 +123,7 @@ size_t abs_persample_stats_bytes(int64_t b, int64_t d);
  *   eta            finite, > 0 (the paper uses 0.05-0.275; values >= 1 are accepted)
  *   b_cur          >= 1, the current global batch size
  *   stats_out      device, abs_stats_bytes(d, n_shards) bytes, 16-byte aligned
- *   gbar_out       device, d floats; must not alias any grads[k]
+ *   gbar_out       device, d floats; must not overlap any grads[k] (ABS_ERR_ALIAS)
  *   b_next_out     device, one int64
  * Non-finite inputs are not an error: the flag is raised and b_next = b_cur.
  */
@@ -180,10 +192,14 @@ int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dty
  * Arguments, results and status codes are those of abs_normtest_adamw, except:
  *   stats_out   device, only (ABS_STATS_HEADER + n_shards*ABS_SHARD_STRIDE) doubles
  *               (header and shard records; no scratch tail), 16-byte aligned
- *   limit       ceil(d/c) + n_shards must not exceed ABS_NOALLOC_MAX_CHUNKS, where c = 8192
- *               for d >= 2^23 and 4096 below (any d up to about 1.07e9); larger problems
- *               return ABS_ERR_TOO_LARGE and launch nothing
- * Results are bit-identical to abs_normtest_adamw on the same inputs.
+ *   limit       the call's chunk count -- the sum over shards of ceil(shard length / c),
+ *               c = 8192 for d >= 2^23 and 4096 below -- must not exceed
+ *               ABS_NOALLOC_MAX_CHUNKS (any d up to about 1.07e9); larger problems return
+ *               ABS_ERR_TOO_LARGE and launch nothing.  abs_noalloc_fits() answers the same
+ *               question on the host without touching the GPU.
+ * Both entry points run the same kernels on the same chunk layout, so on the same inputs
+ * every output (statistics, shard records, b_next, gbar, params, m, v) is bit-identical to
+ * abs_normtest_adamw's.
  *
  * Shared state.  All calls on one device use the same built-in array.  Nothing in it has
  * to be cleared between calls: every record the final reduction reads is written earlier
@@ -194,9 +210,14 @@ int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dty
  * First call.  The first call on each device looks up the device address of the built-in
  * array (cudaGetSymbolAddress, with that device current; this may also trigger the lazy
  * load of the library's device code).  Make that first call outside of any stream
- * capture; later calls on the same device only launch kernels.
+ * capture; later calls on the same device only launch kernels.  The address is cached for
+ * the life of the process: it does not survive cudaDeviceReset() or the destruction of the
+ * device's primary context, after which this entry point must not be used again.
  */
 enum { ABS_NOALLOC_MAX_CHUNKS = 131072 };
+/* 1 if abs_normtest_adamw_noalloc accepts this (d, shard table), 0 if it would return
+ * ABS_ERR_TOO_LARGE or the arguments are invalid.  Host, pure. */
+int abs_noalloc_fits(int64_t d, const int64_t* shard_offsets, int n_shards);
 int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                                const int64_t* shard_offsets, int n_shards, double eta,
                                int64_t b_cur, void* stats_out, float* gbar_out,
@@ -228,6 +249,20 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
  */
 int64_t abs_decide(double S, double n2, double norm, double eta, int64_t b_cur, double* T_out,
                    int* flags_out);
+
+/*
+ * FSDP-Norm across processes (Sec. 3.3; Appendix A: the shard gradients are concatenated, so
+ * the statistic is formed from the sums of all shards).  Each rank runs the norm test on its
+ * own index range and contributes its three sums; every rank then calls this with the
+ * gathered rows and obtains the same bits.
+ *   per_rank    host, n_ranks rows of 3 doubles {n2_r, S_r, Q_r} in rank order
+ *   totals_out  host, 3 doubles {n2, S, Q}: the rows added in rank order (the order in which
+ *               the single-device call adds its shard records); may be NULL
+ * Then the decision of abs_decide on the totals.  Returns b_next, or -1 when per_rank is NULL
+ * or n_ranks < 1.  Pure.
+ */
+int64_t abs_combine_sums(const double* per_rank, int n_ranks, double norm, double eta,
+                         int64_t b_cur, double* totals_out, double* T_out, int* flags_out);
 
 /* Algorithm 1's rounding of a new batch size to the parallel layout:
  * micro = ceil(b/(J*M)), mini = M*micro, returns J*mini.  J, M >= 1.  Returns -1 on

@@ -6,7 +6,7 @@ is its thin Python binding plus the seeded synthetic-input generators.
 from .binding import (ABS_BF16, ABS_F32, ABS_FLAG_DEGENERATE, ABS_FLAG_NONFINITE,  # noqa: F401
                       ABS_FLAG_VIOLATED, AbsError, FusedStep, abs_adamw_hparams, abs_adamw_step, abs_adamw_step_clipped,
                       abs_adamw_step_mixed, abs_normtest_adamw_mixed,
-                      abs_decide,
+                      abs_decide, abs_combine_sums, abs_noalloc_fits,
                       abs_norm_test, abs_normtest_adamw, abs_normtest_adamw_noalloc,
                       abs_persample_norm_test,
                       abs_persample_stats_bytes, abs_round_batch, abs_schedule_advance,

@@ -17,6 +17,7 @@ ABS_OK = 0
 ABS_ERR_NULL, ABS_ERR_RANGE, ABS_ERR_SHARDS, ABS_ERR_ALIGN, ABS_ERR_DTYPE, ABS_ERR_CUDA = (
     -1, -2, -3, -4, -5, -6)
 ABS_ERR_TOO_LARGE = -7
+ABS_ERR_ALIAS = -8
 ABS_NOALLOC_MAX_CHUNKS = 131072
 ABS_MAX_WORKERS, ABS_MAX_SHARDS = 64, 128
 (ABS_STAT_N2, ABS_STAT_S, ABS_STAT_Q, ABS_STAT_T, ABS_STAT_FLAGS, ABS_STAT_NORM,
@@ -77,6 +78,10 @@ def lib():
     L.abs_adamw_step_mixed.argtypes = [ptr, ptr, ptr, ptr, ptr, i64, ptr, i64, dbl, ptr, ptr]
     L.abs_persample_norm_test.restype = cint
     L.abs_persample_norm_test.argtypes = [ptr, i64, i64, i64, cint, dbl, ptr, ptr, ptr, ptr]
+    L.abs_noalloc_fits.restype = cint
+    L.abs_noalloc_fits.argtypes = [i64, ptr, cint]
+    L.abs_combine_sums.restype = i64
+    L.abs_combine_sums.argtypes = [ptr, cint, dbl, dbl, i64, ptr, ptr, ptr]
     L.abs_decide.restype = i64
     L.abs_decide.argtypes = [dbl, dbl, dbl, dbl, i64, ptr, ptr]
     L.abs_round_batch.restype = i64
@@ -109,6 +114,38 @@ def _check_f32_vec(t, d, name):
         raise TypeError("%s must be a contiguous float32 vector of %d elements" % (name, d))
     if not t.is_cuda:
         raise TypeError("%s must live on a CUDA device" % name)
+
+
+def _check_stats(t, nbytes, name="stats_out"):
+    """stats_out must be a CUDA buffer of at least `nbytes` bytes, 16-byte aligned: the kernels
+    write every chunk record (and the per-sample work space) without a bounds check."""
+    if nbytes <= 0:
+        raise ValueError("invalid problem size for %s" % name)
+    if not getattr(t, "is_cuda", False) or not t.is_contiguous():
+        raise TypeError("%s must be a contiguous CUDA tensor" % name)
+    if t.numel() * t.element_size() < nbytes:
+        raise ValueError("%s holds %d bytes, the call needs %d (see abs_stats_bytes)"
+                         % (name, t.numel() * t.element_size(), nbytes))
+    if t.data_ptr() % 16:
+        raise ValueError("%s must be 16-byte aligned" % name)
+
+
+def _check_b_next(t):
+    if (not getattr(t, "is_cuda", False) or t.dtype != torch.int64 or t.numel() < 1
+            or not t.is_contiguous()):
+        raise TypeError("b_next_out must be a CUDA int64 tensor with at least one element")
+
+
+def _check_one_device(*tensors):
+    """All buffers of a call live on the CUDA device that is current: the library launches on
+    the current device and caches per-device kernel attributes under its index."""
+    cur = torch.cuda.current_device()
+    for t in tensors:
+        if t is None:
+            continue
+        if not t.is_cuda or t.device.index != cur:
+            raise ValueError("every buffer must live on the current CUDA device (cuda:%d), got %s"
+                             % (cur, t.device))
 
 
 def _stream(stream):
@@ -176,6 +213,9 @@ def abs_norm_test(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offs
     table, K, d, code = _grad_table(grads)
     offs, n_shards = _offsets(shard_offsets)
     _check_f32_vec(gbar_out, d, "gbar_out")
+    _check_stats(stats_out, abs_stats_bytes(d, n_shards))
+    _check_b_next(b_next_out)
+    _check_one_device(*grads, stats_out, gbar_out, b_next_out)
     rc = lib().abs_norm_test(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
                              stats_out.data_ptr(), gbar_out.data_ptr(), b_next_out.data_ptr(),
                              _stream(stream))
@@ -187,6 +227,7 @@ def abs_adamw_step(params, gbar, m, v, hparams, step, stream=None):
     d = params.numel()
     for t, name in ((params, "params"), (gbar, "gbar"), (m, "m"), (v, "v")):
         _check_f32_vec(t, d, name)
+    _check_one_device(params, gbar, m, v)
     hp = _hparams(hparams)
     rc = lib().abs_adamw_step(params.data_ptr(), gbar.data_ptr(), m.data_ptr(), v.data_ptr(), d,
                               ctypes.byref(hp), int(step), _stream(stream))
@@ -200,6 +241,8 @@ def abs_adamw_step_clipped(params, gbar, m, v, hparams, step, max_norm, stats_in
     d = params.numel()
     for t, name in ((params, "params"), (gbar, "gbar"), (m, "m"), (v, "v")):
         _check_f32_vec(t, d, name)
+    _check_stats(stats_in, 8 * ABS_STATS_HEADER, "stats_in")
+    _check_one_device(params, gbar, m, v, stats_in)
     hp = _hparams(hparams)
     rc = lib().abs_adamw_step_clipped(params.data_ptr(), gbar.data_ptr(), m.data_ptr(),
                                       v.data_ptr(), d, ctypes.byref(hp), int(step),
@@ -216,6 +259,9 @@ def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, param
         _check_f32_vec(t, d, name)
     if gbar_out is not None:
         _check_f32_vec(gbar_out, d, "gbar_out")
+    _check_stats(stats_out, abs_stats_bytes(d, n_shards))
+    _check_b_next(b_next_out)
+    _check_one_device(*grads, stats_out, gbar_out, b_next_out, params, m, v)
     hp = _hparams(hparams)
     rc = lib().abs_normtest_adamw(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
                                   stats_out.data_ptr(),
@@ -243,6 +289,9 @@ def abs_normtest_adamw_mixed(grads, eta, b_cur, stats_out, gbar_out, b_next_out,
     _check_bf16_vec(params_bf16_out, d, "params_bf16_out")
     if gbar_out is not None:
         _check_f32_vec(gbar_out, d, "gbar_out")
+    _check_stats(stats_out, abs_stats_bytes(d, n_shards))
+    _check_b_next(b_next_out)
+    _check_one_device(*grads, stats_out, gbar_out, b_next_out, params, m, v, params_bf16_out)
     hp = _hparams(hparams)
     rc = lib().abs_normtest_adamw_mixed(table, K, d, code, offs, n_shards, float(eta),
                                         int(b_cur), stats_out.data_ptr(),
@@ -262,6 +311,9 @@ def abs_adamw_step_mixed(params, gbar, m, v, params_bf16_out, hparams, step, max
     for t, name in ((params, "params"), (gbar, "gbar"), (m, "m"), (v, "v")):
         _check_f32_vec(t, d, name)
     _check_bf16_vec(params_bf16_out, d, "params_bf16_out")
+    if stats_in is not None:
+        _check_stats(stats_in, 8 * ABS_STATS_HEADER, "stats_in")
+    _check_one_device(params, gbar, m, v, params_bf16_out, stats_in)
     hp = _hparams(hparams)
     rc = lib().abs_adamw_step_mixed(params.data_ptr(), gbar.data_ptr(), m.data_ptr(),
                                     v.data_ptr(), params_bf16_out.data_ptr(), d,
@@ -285,8 +337,9 @@ def abs_normtest_adamw_noalloc(grads, eta, b_cur, stats_out, gbar_out, b_next_ou
         _check_f32_vec(t, d, name)
     if gbar_out is not None:
         _check_f32_vec(gbar_out, d, "gbar_out")
-    if stats_out.numel() * stats_out.element_size() < 8 * (ABS_STATS_HEADER + n_shards * ABS_SHARD_STRIDE):
-        raise ValueError("stats_out is smaller than header + shard records")
+    _check_stats(stats_out, 8 * (ABS_STATS_HEADER + n_shards * ABS_SHARD_STRIDE))
+    _check_b_next(b_next_out)
+    _check_one_device(*grads, stats_out, gbar_out, b_next_out, params, m, v)
     hp = _hparams(hparams)
     rc = lib().abs_normtest_adamw_noalloc(table, K, d, code, offs, n_shards, float(eta),
                                           int(b_cur), stats_out.data_ptr(),
@@ -317,6 +370,9 @@ class FusedStep:
             _check_f32_vec(t, self._d, name)
         if gbar_out is not None:
             _check_f32_vec(gbar_out, self._d, "gbar_out")
+        _check_stats(stats_out, abs_stats_bytes(self._d, self._n_shards))
+        _check_b_next(b_next_out)
+        _check_one_device(*grads, stats_out, gbar_out, b_next_out, params, m, v, params_bf16_out)
         self._hp = _hparams(hparams)
         self._hp_ref = ctypes.byref(self._hp)
         self._ptrs = (stats_out.data_ptr(), gbar_out.data_ptr() if gbar_out is not None else None,
@@ -346,6 +402,9 @@ def abs_persample_norm_test(G, eta, stats_out, gbar_out, b_next_out, stream=None
         raise TypeError("G must be a CUDA matrix [b, d] with unit column stride")
     b, d, ld = G.shape[0], G.shape[1], G.stride(0)
     _check_f32_vec(gbar_out, d, "gbar_out")
+    _check_stats(stats_out, abs_persample_stats_bytes(b, d))
+    _check_b_next(b_next_out)
+    _check_one_device(G, stats_out, gbar_out, b_next_out)
     rc = lib().abs_persample_norm_test(G.data_ptr(), b, d, ld, _dtype_code(G), float(eta),
                                        stats_out.data_ptr(), gbar_out.data_ptr(),
                                        b_next_out.data_ptr(), _stream(stream))
@@ -359,6 +418,26 @@ def abs_decide(S, n2, norm, eta, b_cur):
     b_next = lib().abs_decide(float(S), float(n2), float(norm), float(eta), int(b_cur),
                               ctypes.byref(T), ctypes.byref(flags))
     return int(b_next), T.value, flags.value
+
+
+def abs_combine_sums(rows, norm, eta, b_cur):
+    """rows: one (n2, S, Q) triple per rank, in rank order.  Returns a dict with the totals
+    (added in rank order by the library), T, flags and b_next."""
+    n = len(rows)
+    flat = (ctypes.c_double * (3 * n))(*[float(x) for row in rows for x in row])
+    tot = (ctypes.c_double * 3)()
+    T, flags = ctypes.c_double(0.0), ctypes.c_int(0)
+    b_next = lib().abs_combine_sums(flat, n, float(norm), float(eta), int(b_cur), tot,
+                                    ctypes.byref(T), ctypes.byref(flags))
+    if b_next < 0:
+        raise ValueError("abs_combine_sums rejected its arguments")
+    return {"n2": tot[0], "S": tot[1], "Q": tot[2], "T": T.value, "flags": flags.value,
+            "b_next": int(b_next)}
+
+
+def abs_noalloc_fits(d, shard_offsets=None):
+    offs, n_shards = _offsets(shard_offsets)
+    return bool(lib().abs_noalloc_fits(int(d), offs, n_shards))
 
 
 def abs_round_batch(b_next, J, M):

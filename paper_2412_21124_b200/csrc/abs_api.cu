@@ -80,10 +80,50 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStre
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// Largest cluster (8, 4, 2 or 1 CTAs) of finalize_kernel that the current device can
+// co-schedule, asked once per device and cached.  A refusal (SM partitioning, a shared
+// device) or a failing query means 1: a plain single-CTA launch, which cannot be refused for
+// lack of co-scheduling.  The sums do not depend on the cluster size, so the fallback changes
+// no output bit.
+int finalize_max_cluster() {
+  static std::mutex mu;
+  static int cached[64] = {};  // 0 = not asked yet
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev]) return cached[dev];
+  }
+  int best = 1;
+  for (int n = kFinalizeMaxCtas; n > 1; n /= 2) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n);
+    cfg.blockDim = dim3(kFinalizeThreads);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = n;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int active = 0;
+    if (cudaOccupancyMaxActiveClusters(&active, finalize_kernel, &cfg) == cudaSuccess &&
+        active >= 1) {
+      best = n;
+      break;
+    }
+  }
+  (void)cudaGetLastError();  // a refused query is an answer, not an error of the call
+  std::lock_guard<std::mutex> lock(mu);
+  cached[dev] = best;
+  return best;
+}
+
 // The finalize kernel runs as one thread-block cluster.  The slice size (and with it the
 // shape of every sum) follows from the chunk counts alone; the cluster size only decides how
-// many warps share the slices.
-cudaError_t launch_finalize(FinalizeParams fp, cudaStream_t st) {
+// many warps share the slices.  `max_ctas` is finalize_max_cluster(), queried by the caller
+// before its first launch so that nothing that can be foreseen fails after it.
+cudaError_t launch_finalize(FinalizeParams fp, int max_ctas, cudaStream_t st) {
   int slice = kFinalizeSlice;
   for (;;) {
     int64_t n = 0;
@@ -99,7 +139,8 @@ cudaError_t launch_finalize(FinalizeParams fp, cudaStream_t st) {
         fp.slice_prefix[s] + (fp.chunk_prefix[s + 1] - fp.chunk_prefix[s] + slice - 1) / slice;
   const int n_slices = fp.slice_prefix[fp.n_shards];
   unsigned n_ctas = 1;
-  while (n_ctas < kFinalizeMaxCtas && static_cast<int>(n_ctas) * kFinalizeSlicesPerCta < n_slices)
+  while (static_cast<int>(n_ctas) < max_ctas &&
+         static_cast<int>(n_ctas) * kFinalizeSlicesPerCta < n_slices)
     n_ctas *= 2;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_ctas);
@@ -114,12 +155,36 @@ cudaError_t launch_finalize(FinalizeParams fp, cudaStream_t st) {
   attr[1].val.clusterDim.y = 1;
   attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 2;
+  cfg.numAttrs = n_ctas > 1 ? 2 : 1;  // one CTA: an ordinary launch (its own implicit cluster)
   return cudaLaunchKernelEx(&cfg, finalize_kernel, fp);
 }
 
 bool misaligned(const void* p, size_t a) {
   return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
+}
+
+// [a, a+na) and [b, b+nb) share a byte
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+  return a0 < b0 + nb && b0 < a0 + na;
+}
+
+// Aliasing rule of the norm-test calls: no output range may share a byte with a gradient
+// buffer or with another output (the kernels read every input coordinate exactly once and
+// give no ordering between a chunk's reads and another chunk's writes).
+struct Range {
+  const void* p;
+  size_t bytes;
+};
+bool any_alias(const void* const* grads, int K, size_t grad_bytes, const Range* outs, int n_outs) {
+  for (int i = 0; i < n_outs; ++i) {
+    if (!outs[i].p) continue;
+    for (int k = 0; k < K; ++k)
+      if (overlaps(outs[i].p, outs[i].bytes, grads[k], grad_bytes)) return true;
+    for (int j = i + 1; j < n_outs; ++j)
+      if (outs[j].p && overlaps(outs[i].p, outs[i].bytes, outs[j].p, outs[j].bytes)) return true;
+  }
+  return false;
 }
 
 struct Layout {
@@ -300,11 +365,44 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// abs_normtest_adamw_noalloc: the fused step with its chunk records in an array that is
+// part of the library image, for callers that cannot allocate device memory.
+// ---------------------------------------------------------------------------------------
+// One {n2, S, Q, 0} record per chunk.  Lives in every device's copy of the module.
+static __device__ __align__(256) double g_noalloc_chunk_records[ABS_NOALLOC_MAX_CHUNKS * 4];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+double* g_noalloc_device_ptr[kMaxDevices] = {};  // device address of the array, per device
+
+// In host code `g_noalloc_chunk_records` is only a handle for the runtime, not an address
+// a kernel could use: the device address is looked up once per device (with that device
+// current) and cached.
+int noalloc_records_for_current_device(double** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= kMaxDevices) return ABS_ERR_RANGE;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_device_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_chunk_records);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_noalloc_device_ptr[dev] = static_cast<double*>(p);
+  }
+  *out = g_noalloc_device_ptr[dev];
+  return ABS_OK;
+}
+
+// The one body behind abs_norm_test, abs_normtest_adamw(_mixed) and the no-alloc variant.
+// `builtin_records`: the per-chunk records go to the array built into the library (no-alloc
+// variant; stats_out is then header + shard records only) instead of the tail of stats_out.
 int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                   const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
                   void* stats_out, float* gbar_out, int64_t* b_next_out, float* params, float* m,
                   float* v, void* params_bf16, const abs_adamw_hparams* hparams, int64_t step,
-                  bool fused, abs_stream_t stream) {
+                  bool fused, abs_stream_t stream, bool builtin_records = false) {
   if (!grads || !stats_out || !b_next_out) return ABS_ERR_NULL;
   if (!fused && !gbar_out) return ABS_ERR_NULL;
   if (fused && (!params || !m || !v)) return ABS_ERR_NULL;
@@ -329,10 +427,29 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   Layout L;
   const int rc = make_layout(d, shard_offsets, n_shards, fused, &L);
   if (rc != ABS_OK) return rc;
+  if (builtin_records && L.n_chunks > ABS_NOALLOC_MAX_CHUNKS) return ABS_ERR_TOO_LARGE;
 
+  const size_t ud = static_cast<size_t>(d);
+  const size_t stats_bytes =
+      builtin_records
+          ? sizeof(double) * (ABS_STATS_HEADER + static_cast<size_t>(L.n_shards) * ABS_SHARD_STRIDE)
+          : abs_stats_bytes(d, L.n_shards);
+  const Range outs[] = {{gbar_out, ud * 4}, {params, ud * 4},       {m, ud * 4},
+                        {v, ud * 4},        {params_bf16, ud * 2},  {stats_out, stats_bytes},
+                        {b_next_out, 8}};
+  if (any_alias(grads, K, ud * esz, outs, 7)) return ABS_ERR_ALIAS;
+
+  // everything that can be refused is asked before the first launch
+  const int finalize_ctas = finalize_max_cluster();
   double* stats = static_cast<double*>(stats_out);
   double* chunk_out =
       stats + ABS_STATS_HEADER + static_cast<size_t>(L.n_shards) * ABS_SHARD_STRIDE;
+  if (builtin_records) {
+    // every record the final reduction reads is written by this call's first kernel, so the
+    // previous call's contents of the shared array are never observed
+    const int rc2 = noalloc_records_for_current_device(&chunk_out);
+    if (rc2 != ABS_OK) return rc2;
+  }
 
   StreamParams prm;
   std::memset(&prm, 0, sizeof prm);
@@ -374,7 +491,7 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   fp.eta = eta;
   fp.norm = static_cast<double>(K);
   fp.b_cur = b_cur;
-  e = launch_finalize(fp, st);
+  e = launch_finalize(fp, finalize_ctas, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -532,6 +649,11 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
   const int64_t nrb = (b + rpb - 1) / rpb;
   if (n_chunks64 > INT32_MAX || nrb > 65535) return ABS_ERR_RANGE;
 
+  if (overlaps(G, static_cast<size_t>(b - 1) * ld * 4 + static_cast<size_t>(d) * 4, gbar_out,
+               static_cast<size_t>(d) * 4))
+    return ABS_ERR_ALIAS;
+  const int finalize_ctas = finalize_max_cluster();
+
   double* stats = static_cast<double*>(stats_out);
   PersampleParams prm;
   std::memset(&prm, 0, sizeof prm);
@@ -576,7 +698,7 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
   fp.eta = eta;
   fp.norm = static_cast<double>(b - 1);
   fp.b_cur = b;
-  e = launch_finalize(fp, st);
+  e = launch_finalize(fp, finalize_ctas, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -600,6 +722,21 @@ int64_t abs_decide(double S, double n2, double norm, double eta, int64_t b_cur, 
   return b_next;
 }
 
+int64_t abs_combine_sums(const double* per_rank, int n_ranks, double norm, double eta,
+                         int64_t b_cur, double* totals_out, double* T_out, int* flags_out) {
+  if (!per_rank || n_ranks < 1) {
+    if (T_out) *T_out = std::nan("");
+    if (flags_out) *flags_out = 0;
+    return -1;
+  }
+  double tot[3] = {0.0, 0.0, 0.0};
+  for (int r = 0; r < n_ranks; ++r)  // rank order, the order in which shard records are added
+    for (int j = 0; j < 3; ++j) tot[j] += per_rank[3 * r + j];
+  if (totals_out)
+    for (int j = 0; j < 3; ++j) totals_out[j] = tot[j];
+  return abs_decide(tot[1], tot[0], norm, eta, b_cur, T_out, flags_out);
+}
+
 int64_t abs_round_batch(int64_t b_next, int64_t J, int64_t M) {
   if (b_next < 1 || J < 1 || M < 1) return -1;
   const int64_t jm = J * M;
@@ -619,6 +756,8 @@ const char* abs_status_string(int status) {
     case ABS_ERR_TOO_LARGE:
       return "the problem needs more chunk records than the built-in scratch holds "
              "(ABS_NOALLOC_MAX_CHUNKS); use abs_normtest_adamw with a caller-sized stats_out";
+    case ABS_ERR_ALIAS:
+      return "an output buffer overlaps a gradient buffer or another output buffer";
     default: return "unknown status";
   }
 }
@@ -627,109 +766,24 @@ int abs_last_cuda_error(void) { return g_last_cuda_error; }
 
 }  // extern "C"
 
-// ---------------------------------------------------------------------------------------
-// abs_normtest_adamw_noalloc: the fused step with its chunk records in an array that is
-// part of the library image, for callers that cannot allocate device memory.
-// ---------------------------------------------------------------------------------------
-namespace {
+extern "C" {
 
-// One {n2, S, Q, 0} record per chunk.  Lives in every device's copy of the module.
-static __device__ __align__(256) double g_noalloc_chunk_records[ABS_NOALLOC_MAX_CHUNKS * 4];
-
-constexpr int kMaxDevices = 64;
-std::mutex g_noalloc_mutex;
-double* g_noalloc_device_ptr[kMaxDevices] = {};  // device address of the array, per device
-
-// In host code `g_noalloc_chunk_records` is only a handle for the runtime, not an address
-// a kernel could use: the device address is looked up once per device (with that device
-// current) and cached.
-int noalloc_records_for_current_device(double** out) {
-  int dev = -1;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return cuda_fail(e);
-  if (dev < 0 || dev >= kMaxDevices) return ABS_ERR_RANGE;
-  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
-  if (!g_noalloc_device_ptr[dev]) {
-    void* p = nullptr;
-    e = cudaGetSymbolAddress(&p, g_noalloc_chunk_records);
-    if (e != cudaSuccess) return cuda_fail(e);
-    g_noalloc_device_ptr[dev] = static_cast<double*>(p);
-  }
-  *out = g_noalloc_device_ptr[dev];
-  return ABS_OK;
-}
-
-}  // namespace
-
-extern "C" int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64_t d,
-                                          abs_dtype dtype, const int64_t* shard_offsets,
-                                          int n_shards, double eta, int64_t b_cur,
-                                          void* stats_out, float* gbar_out, int64_t* b_next_out,
-                                          float* params, float* m, float* v,
-                                          const abs_adamw_hparams* hparams, int64_t step,
-                                          abs_stream_t stream) {
-  if (!grads || !stats_out || !b_next_out || !params || !m || !v) return ABS_ERR_NULL;
-  if (dtype != ABS_F32 && dtype != ABS_BF16) return ABS_ERR_DTYPE;
-  if (K < 1 || K > ABS_MAX_WORKERS || d < 1 || b_cur < 1) return ABS_ERR_RANGE;
-  if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
-  int rc = check_hparams(hparams, step);
-  if (rc != ABS_OK) return rc;
-  const size_t esz = (dtype == ABS_F32) ? 4 : 2;
-  for (int k = 0; k < K; ++k) {
-    if (!grads[k]) return ABS_ERR_NULL;
-    if (misaligned(grads[k], esz)) return ABS_ERR_ALIGN;
-  }
-  if (misaligned(stats_out, 16) || misaligned(b_next_out, 8)) return ABS_ERR_ALIGN;
-  if (gbar_out && misaligned(gbar_out, 4)) return ABS_ERR_ALIGN;
-  if (misaligned(params, 4) || misaligned(m, 4) || misaligned(v, 4)) return ABS_ERR_ALIGN;
-
+int abs_noalloc_fits(int64_t d, const int64_t* shard_offsets, int n_shards) {
+  if (d < 1) return 0;
   Layout L;
-  rc = make_layout(d, shard_offsets, n_shards, true, &L);
-  if (rc != ABS_OK) return rc;
-  if (L.n_chunks > ABS_NOALLOC_MAX_CHUNKS) return ABS_ERR_TOO_LARGE;
-
-  double* records = nullptr;
-  rc = noalloc_records_for_current_device(&records);
-  if (rc != ABS_OK) return rc;
-
-  StreamParams prm;
-  std::memset(&prm, 0, sizeof prm);
-  for (int k = 0; k < K; ++k) prm.grads[k] = grads[k];
-  std::memcpy(prm.shard_off, L.shard_off, sizeof(int64_t) * (L.n_shards + 1));
-  std::memcpy(prm.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
-  prm.d = d;
-  prm.K = K;
-  prm.n_shards = L.n_shards;
-  prm.n_chunks = L.n_chunks;
-  prm.chunk_elems = L.chunk_elems;
-  prm.inv_K = 1.0 / static_cast<double>(K);
-  prm.inv_Kf = static_cast<float>(prm.inv_K);
-  prm.neg_Kf = -static_cast<float>(K);
-  prm.gbar = gbar_out;
-  prm.p = params;
-  prm.m = m;
-  prm.v = v;
-  prm.chunk_out = records;  // every record read below is written by this launch first
-  prm.adam = make_adam(hparams, step);
-
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  cudaError_t e = (dtype == ABS_F32) ? launch_stream<F32, true>(prm, st)
-                                     : launch_stream<BF16, true>(prm, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-
-  FinalizeParams fp;
-  std::memset(&fp, 0, sizeof fp);
-  fp.chunk_in = records;
-  std::memcpy(fp.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
-  fp.n_shards = L.n_shards;
-  fp.n_chunks = L.n_chunks;
-  fp.stats = static_cast<double*>(stats_out);
-  fp.b_next = b_next_out;
-  fp.eta = eta;
-  fp.norm = static_cast<double>(K);
-  fp.b_cur = b_cur;
-  e = launch_finalize(fp, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-  return ABS_OK;
+  if (make_layout(d, shard_offsets, n_shards, true, &L) != ABS_OK) return 0;
+  return L.n_chunks <= ABS_NOALLOC_MAX_CHUNKS ? 1 : 0;
 }
 
+int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                               const int64_t* shard_offsets, int n_shards, double eta,
+                               int64_t b_cur, void* stats_out, float* gbar_out,
+                               int64_t* b_next_out, float* params, float* m, float* v,
+                               const abs_adamw_hparams* hparams, int64_t step,
+                               abs_stream_t stream) {
+  return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
+                       gbar_out, b_next_out, params, m, v, nullptr, hparams, step, true, stream,
+                       /*builtin_records=*/true);
+}
+
+}  // extern "C"

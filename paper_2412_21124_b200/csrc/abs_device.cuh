@@ -163,6 +163,16 @@ __device__ __forceinline__ void adamw_pair(const AdamScalars& a, float2 g, float
   const float2 upd = __fmul2_rn(__fmul2_rn(make_float2(a.step_size, a.step_size), m), inv);
   w = __ffma2_rn(make_float2(a.decay, a.decay), w, make_float2(-upd.x, -upd.y));
 }
+// max(x, +0) that keeps a NaN: the shifted one-pass variance can come out a few ulps below
+// zero and is clamped, but a NaN (a non-finite input, or squares that overflowed to inf - inf)
+// has to reach the sums so that the call reports ABS_FLAG_NONFINITE.  fmaxf would return 0.
+__device__ __forceinline__ float clamp_nonneg(float x) {
+  float r;
+  asm("max.NaN.f32 %0, %1, 0f00000000;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ double clamp_nonneg(double x) { return x < 0.0 ? 0.0 : x; }
+
 // Mean of K fp32 partial sums: s/K.  For K a power of two the product with 1/K is exact;
 // otherwise one residual correction makes K identical inputs return exactly that input.
 template <bool POW2>

@@ -112,7 +112,7 @@ __device__ __forceinline__ float coord_math_split(const float (&g)[KB], int K,
     }
   const float mean = GT::template mean<false>(s, prm);
   const float dm = mean - c;
-  dev2 = fmaxf(fmaf(prm.neg_Kf * dm, dm, s2), 0.f);
+  dev2 = clamp_nonneg(fmaf(prm.neg_Kf * dm, dm, s2));
   return mean;
 }
 
@@ -521,8 +521,8 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
         gb[2 * pi + 1] = mean.y;
         row_n2 = fmaf(mean.x, mean.x, row_n2);
         row_n2 = fmaf(mean.y, mean.y, row_n2);
-        row_S += fmaxf(t.x, 0.f);
-        row_S += fmaxf(t.y, 0.f);
+        row_S += clamp_nonneg(t.x);
+        row_S += clamp_nonneg(t.y);
         row_Q += q[pi].x;
         row_Q += q[pi].y;
         if (ADAM) adamw_pair(prm.adam, mean, w2[pi], m2[pi], v2[pi]);
@@ -631,6 +631,11 @@ __global__ void __launch_bounds__(kFinalizeThreads)
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   double* part0 = cluster.map_shared_rank(part, 0);
   const int n_slices = fp.slice_prefix[fp.n_shards];
+  // Distributed shared memory of another CTA may only be touched once that CTA is known to
+  // have started: every CTA of the cluster arrives here before the first remote store below.
+  // The barrier touches no global memory, so it sits before the dependency wait and overlaps
+  // the tail of the preceding kernel.
+  cluster.sync();
   grid_dependency_wait();
   for (int i = rank * kFinalizeWarps + warp; i < n_slices; i += n_warps) {
     // the shard of slice i: the last s with slice_prefix[s] <= i

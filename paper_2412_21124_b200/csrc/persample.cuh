@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(kPsThreads, 3)
       // so that identical rows give their common value exactly
       const double mu = (ng == kGroup) ? sum * (1.0 / kGroup) : sum / dn;
       const double dc = mu - static_cast<double>(g.c[i]);
-      const double m2g = fmax(static_cast<double>(g.s2[i]) - dn * dc * dc, 0.0);
+      const double m2g = clamp_nonneg(static_cast<double>(g.s2[i]) - dn * dc * dc);
       const double delta = mu - mean[i];
       mean[i] += delta * w_mean;
       m2[i] += m2g + delta * delta * w_m2;

@@ -6,9 +6,9 @@ the flat vector (the FSDP layout of Sec. 3.3) and only the three fp64 sums per r
 cross the wire.  This module holds that small host-side logic:
 
   rank_range          the contiguous index range a rank owns
-  combine_rank_sums   all-gather of {n2, S, Q} per rank, added in rank order on every
-                      rank (so all ranks take the same bit-identical decision), then the
-                      library's host-side decision
+  combine_rank_sums   all-gather of {n2, S, Q} per rank; the rank-ordered sum and the
+                      decision are the library's abs_combine_sums, called with the same
+                      rows on every rank (so all ranks take the same bit-identical decision)
   sharded_normtest_adamw
                       the fused step on this rank's index range followed by that exchange:
                       the multi-GPU form of FSDP-Norm (Sec. 3.3; Algorithm 1 with the shard
@@ -58,13 +58,8 @@ def combine_rank_sums(n2, S, Q, K, eta, b_cur, device="cpu", group=None):
         dist.all_gather(parts, local, group=group)
     else:
         parts = [local]
-    tot = [0.0, 0.0, 0.0]
-    for part in parts:  # rank order
-        vals = part.tolist()
-        for j in range(3):
-            tot[j] += vals[j]
-    b_next, T, flags = binding.abs_decide(tot[1], tot[0], K, eta, b_cur)
-    return {"n2": tot[0], "S": tot[1], "Q": tot[2], "T": T, "flags": flags, "b_next": b_next}
+    # the rank-ordered sum and the decision are the library's (abs_combine_sums)
+    return binding.abs_combine_sums([part.tolist() for part in parts], K, eta, b_cur)
 
 
 def _gather_rank_rows(local, group=None):
@@ -97,12 +92,7 @@ def sharded_normtest_adamw(grads_local, eta, b_cur, stats_out, gbar_out, b_next_
     binding.abs_normtest_adamw(grads_local, eta, b_cur, stats_out, gbar_out, b_next_out,
                                params_local, m_local, v_local, hparams, step)
     local = stats_out.view(torch.float64)[binding.ABS_STAT_N2:binding.ABS_STAT_Q + 1]
-    tot = [0.0, 0.0, 0.0]
-    for row in _gather_rank_rows(local, group):  # rank order
-        for j in range(3):
-            tot[j] += row[j]
-    b_next, T, flags = binding.abs_decide(tot[1], tot[0], len(grads_local), eta, b_cur)
-    return {"n2": tot[0], "S": tot[1], "Q": tot[2], "T": T, "flags": flags, "b_next": b_next}
+    return binding.abs_combine_sums(_gather_rank_rows(local, group), len(grads_local), eta, b_cur)
 
 
 def barrier(device=None):

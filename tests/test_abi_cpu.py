@@ -1,16 +1,39 @@
 """CPU-side checks of the C ABI: the library loads, exports every declared symbol, its
 host helpers agree with the hand-worked fixtures, and every invalid-argument path returns
-its status before anything could be launched (no GPU is touched here)."""
+its status before anything could be launched.
+
+The reject cases hand fabricated addresses to launching entry points.  They are safe because
+every check comes before the first launch -- and, so that this does not rest on every check
+being right, the whole module runs with CUDA_VISIBLE_DEVICES set to the empty string: the
+library initialises CUDA lazily, on its first runtime call, so with no device visible a launch
+that slipped through a regressed check returns ABS_ERR_CUDA (and fails the test) instead of
+running on an unmapped address."""
 import ctypes
 import json
 import math
 import os
 import re
+import subprocess
+import sys
 
 import pytest
 
 import __graft_entry__ as entry
 from paper_2412_21124_b200 import binding
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _no_visible_device():
+    """Hide every GPU from the CUDA runtime for the life of this module.  The variable is read
+    when the runtime initialises, which nothing here triggers when all checks hold; it is put
+    back afterwards for the modules that follow."""
+    old = os.environ.get("CUDA_VISIBLE_DEVICES")
+    os.environ["CUDA_VISIBLE_DEVICES"] = ""
+    yield
+    if old is None:
+        os.environ.pop("CUDA_VISIBLE_DEVICES", None)
+    else:
+        os.environ["CUDA_VISIBLE_DEVICES"] = old
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 HEADER = os.path.join(ROOT, "include", "abs_normtest.h")
@@ -134,11 +157,11 @@ def test_schedule_rejects(L):
 
 def test_status_strings(L):
     seen = set()
-    for s in range(0, -7, -1):
+    for s in range(0, -9, -1):
         msg = L.abs_status_string(s).decode()
         assert msg and msg != "unknown status"
         seen.add(msg)
-    assert len(seen) == 7
+    assert len(seen) == 9
     assert L.abs_status_string(-99).decode() == "unknown status"
     assert L.abs_last_cuda_error() == 0
 
@@ -320,6 +343,158 @@ def test_adamw_rejects_pointers(L):
 ])
 def test_persample_rejects(L, args, status):
     assert L.abs_persample_norm_test(*args) == status
+
+
+# ---- aliasing: outputs may not overlap the gradients or each other ------------------------
+def _fused_args(table, K, d, dtype, stats, gbar, b_next, p, m, v):
+    hp = _hp()
+    return [table, K, d, dtype, None, 1, 0.1, 8, stats, gbar, b_next, p, m, v, ctypes.byref(hp), 1,
+            None], hp
+
+
+def test_overlapping_buffers_are_rejected(L):
+    d = 1000                       # fp32: 4000 bytes per buffer
+    A = 0x100000                   # fabricated, 16-byte aligned, never dereferenced
+    g0, g1 = A, A + 0x10000
+    stats, b_next = A + 0x80000, A + 0x90000
+    table = (ctypes.c_void_p * 2)(g0, g1)
+    ok_gbar = A + 0x20000
+    nt = lambda gbar, st=stats, bn=b_next: L.abs_norm_test(table, 2, d, 0, None, 1, 0.1, 8, st,
+                                                           gbar, bn, None)
+    # gbar_out inside, at the start of, or straddling the end of a gradient buffer
+    for gbar in (g0, g1, g0 + 4 * (d - 1), g1 - 4 * (d - 1), g0 + 2000):
+        assert nt(gbar) == binding.ABS_ERR_ALIAS, hex(gbar)
+    # stats_out or b_next_out inside a gradient buffer or inside gbar_out
+    assert nt(ok_gbar, st=g1 + 16) == binding.ABS_ERR_ALIAS
+    assert nt(ok_gbar, bn=ok_gbar + 8) == binding.ABS_ERR_ALIAS
+    assert nt(ok_gbar, st=ok_gbar + 4 * d - 16) == binding.ABS_ERR_ALIAS
+    # fused: params/m/v against the gradients, gbar_out and each other
+    p, m, v = A + 0x30000, A + 0x40000, A + 0x50000
+    for bad in (dict(p=g0), dict(m=g1 + 4), dict(v=p), dict(m=p + 4 * (d - 1)), dict(gbar=v),
+                dict(gbar=g0 + 400)):
+        a = dict(p=p, m=m, v=v, gbar=ok_gbar)
+        a.update(bad)
+        args, hp = _fused_args(table, 2, d, 0, stats, a["gbar"], b_next, a["p"], a["m"], a["v"])
+        assert L.abs_normtest_adamw(*args) == binding.ABS_ERR_ALIAS, bad
+        assert L.abs_normtest_adamw_noalloc(*args) == binding.ABS_ERR_ALIAS, bad
+    # the bf16 copy of the parameters (2-byte elements) against a gradient and against params
+    for p16 in (g1 + 2 * (2 * d - 1), p + 4 * d - 2):
+        args, hp = _fused_args(table, 2, d, 0, stats, ok_gbar, b_next, p, m, v)
+        assert L.abs_normtest_adamw_mixed(*(args[:14] + [p16] + args[14:])) == binding.ABS_ERR_ALIAS
+    # (ranges that merely touch are accepted: see test_cuda_failure_is_a_status_not_a_crash)
+    # per-sample: gbar_out inside the matrix
+    assert L.abs_persample_norm_test(A, 4, 10, 12, 0, 0.1, stats, A + 4 * 40, b_next,
+                                     None) == binding.ABS_ERR_ALIAS
+
+
+def test_combine_sums_adds_in_rank_order_and_decides(L):
+    # three ranks whose sums only add up exactly in one order: 1e16 + 1 + 1 differs from
+    # 1 + 1 + 1e16 in fp64
+    rows = [(1e16, 2.0, 0.0), (1.0, 1.0, 0.0), (1.0, 1.0, 0.0)]
+    out = binding.abs_combine_sums(rows, 2, 0.25, 3)
+    assert out["n2"] == (1e16 + 1.0) + 1.0 == 1e16 and out["S"] == 4.0
+    out = binding.abs_combine_sums(rows[::-1], 2, 0.25, 3)
+    assert out["n2"] == (1.0 + 1.0) + 1e16 == 1e16 + 2.0
+    # hand case H1 split over two ranks (coordinate 0 on rank 0, coordinate 1 on rank 1)
+    c = json.load(open(GOLDEN))["norm_test"][0]
+    assert c["n2"] == 8 and c["S"] == 4
+    out = binding.abs_combine_sums([(4.0, 2.0, 10.0), (4.0, 2.0, 10.0)], 2, c["eta"], 3)
+    assert (out["n2"], out["S"], out["Q"], out["T"], out["b_next"]) == (8.0, 4.0, 20.0, 4.0, 4)
+    assert out["flags"] == binding.ABS_FLAG_VIOLATED
+    b, T, flags = binding.abs_decide(4.0, 8.0, 2, c["eta"], 3)
+    assert (b, T, flags) == (out["b_next"], out["T"], out["flags"])
+    # a non-finite rank poisons the decision, the batch size is kept
+    out = binding.abs_combine_sums([(4.0, 2.0, 0.0), (math.nan, 2.0, 0.0)], 2, 0.25, 3)
+    assert out["flags"] == binding.ABS_FLAG_NONFINITE and out["b_next"] == 3
+    assert L.abs_combine_sums(None, 2, 2.0, 0.25, 3, None, None, None) == -1
+    one = (ctypes.c_double * 3)(1.0, 1.0, 1.0)
+    assert L.abs_combine_sums(one, 0, 2.0, 0.25, 3, None, None, None) == -1
+
+
+def test_noalloc_size_limit_is_a_host_check(L):
+    """Problems that would not fit the array built into the library are refused before anything
+    touches the GPU; abs_noalloc_fits answers the same question."""
+    cap = binding.ABS_NOALLOC_MAX_CHUNKS
+    assert binding.abs_noalloc_fits(1)
+    assert binding.abs_noalloc_fits(cap * 8192)            # exactly the capacity
+    assert not binding.abs_noalloc_fits(cap * 8192 + 1)
+    assert not binding.abs_noalloc_fits(0)
+    # shard cuts add ragged chunks: the same d no longer fits when every shard ends mid-chunk
+    d = cap * 8192 - 5
+    assert binding.abs_noalloc_fits(d)
+    assert not binding.abs_noalloc_fits(d, [0, 1, 2, d])
+    assert not binding.abs_noalloc_fits(100, [0, 50, 40, 100])   # invalid table
+    table = (ctypes.c_void_p * 2)(FAKE, FAKE + 0x1000)
+    hp = _hp()
+    big = 1 << 50  # fabricated, far apart: the alias check is passed on the way
+    rc = L.abs_normtest_adamw_noalloc(table, 2, cap * 8192 + 1, binding.ABS_BF16, None, 1, 0.1, 8,
+                                      big, None, big + 64, 2 * big, 3 * big, 4 * big,
+                                      ctypes.byref(hp), 1, None)
+    assert rc == binding.ABS_ERR_TOO_LARGE
+    assert "ABS_NOALLOC_MAX_CHUNKS" in L.abs_status_string(rc).decode()
+
+
+class _FakeCudaTensor:
+    """Just enough of a tensor for the binding's buffer checks (no GPU here)."""
+    is_cuda = True
+
+    def __init__(self, nbytes, ptr=0x10000, itemsize=8):
+        self._n, self._ptr, self._sz = nbytes // itemsize, ptr, itemsize
+
+    def numel(self):
+        return self._n
+
+    def element_size(self):
+        return self._sz
+
+    def is_contiguous(self):
+        return True
+
+    def data_ptr(self):
+        return self._ptr
+
+
+def test_binding_refuses_short_or_misplaced_stats_buffers(L):
+    need = binding.abs_stats_bytes(1 << 20, 4)
+    binding._check_stats(_FakeCudaTensor(need), need)
+    with pytest.raises(ValueError, match="abs_stats_bytes"):
+        binding._check_stats(_FakeCudaTensor(need - 8), need)
+    # a header-only buffer (what the no-alloc call takes) handed to the plain call
+    with pytest.raises(ValueError):
+        binding._check_stats(_FakeCudaTensor(8 * (binding.ABS_STATS_HEADER + 4 * 4)), need)
+    with pytest.raises(ValueError, match="aligned"):
+        binding._check_stats(_FakeCudaTensor(need, ptr=0x10008), need)
+    import torch
+    with pytest.raises(TypeError):
+        binding._check_stats(torch.zeros(need // 8, dtype=torch.float64), need)  # host memory
+    with pytest.raises(TypeError):
+        binding._check_b_next(torch.zeros(1, dtype=torch.int64))
+    with pytest.raises(ValueError):
+        binding._check_stats(_FakeCudaTensor(64), 0)
+
+
+def test_cuda_failure_is_a_status_not_a_crash():
+    """Valid arguments but no usable device: the first runtime call fails, the entry point
+    returns ABS_ERR_CUDA, abs_last_cuda_error holds the code, nothing ran.  In a child process,
+    so that the failed initialisation stays out of this one."""
+    code = (
+        "import ctypes, sys\n"
+        "sys.path.insert(0, %r)\n"
+        "from paper_2412_21124_b200 import binding as B\n"
+        "L = B.lib()\n"
+        "hp = B.abs_adamw_hparams(1e-3, 0.9, 0.999, 1e-8, 0.1)\n"
+        "A = 0x100000\n"
+        "rc = L.abs_adamw_step(A, A + 0x10000, A + 0x20000, A + 0x30000, 100, ctypes.byref(hp), 1, None)\n"
+        "print(rc, L.abs_last_cuda_error())\n"
+        "# buffers that touch end to start do not overlap: the alias check lets them through\n"
+        "d = 1000\n"
+        "table = (ctypes.c_void_p * 2)(A, A + 2 * d)\n"
+        "rc = L.abs_norm_test(table, 2, d, 1, None, 1, 0.1, 8, A + 0x80000, A + 4 * d, A + 0x90000, None)\n"
+        "print(rc, L.abs_last_cuda_error())\n" % ROOT)
+    env = dict(os.environ, CUDA_VISIBLE_DEVICES="")
+    out = subprocess.check_output([sys.executable, "-c", code], env=env).decode().split()
+    assert int(out[0]) == binding.ABS_ERR_CUDA and int(out[1]) != 0
+    assert int(out[2]) == binding.ABS_ERR_CUDA and int(out[3]) != 0
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
