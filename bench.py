@@ -19,7 +19,6 @@ import os
 import re
 import statistics
 import sys
-import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -34,6 +33,8 @@ GRAD_BYTES = 2           # bf16
 BYTES_PER_ELEM = K_WORKERS * GRAD_BYTES + 24   # K*s read + p,m,v read and written
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
+TIMED_REGION_MS = 1000.0   # the timed blocks together last about this long ...
+MIN_BLOCKS, MAX_BLOCKS = 3, 400   # ... but there are at least 3 and at most 400 of them
 
 
 def workload_config(d):
@@ -53,12 +54,16 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+FUSED_KERNEL_SOURCES = ("abs_device.cuh", "normtest_bulk.cuh", "normtest_stream.cuh")
+
+
 def kernel_source_hash():
-    """Hash of the kernel sources as the compiler sees them: comments, blank lines and
-    indentation do not count (no string literal in those files contains a comment marker)."""
+    """Hash of the sources the fused kernel is compiled from, as the compiler sees them:
+    comments, blank lines and indentation do not count (no string literal in those files
+    contains a comment marker)."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2412_21124_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
+    for name in FUSED_KERNEL_SOURCES:
         with open(os.path.join(csrc, name), "r", encoding="utf-8") as f:
             text = f.read()
         text = re.sub(r"/\*.*?\*/", " ", text, flags=re.S)
@@ -72,76 +77,27 @@ def kernel_source_hash():
 
 
 def recorded_traffic(d):
-    """DRAM bytes per launch of the fused kernel from the committed ncu summary, or None
-    when the kernel sources changed after the counters were taken."""
+    """DRAM bytes per launch of the fused kernel from the committed ncu counters, or None when
+    the kernel sources changed after the counters were taken.  The record holds the counters
+    of launches at `d_measured` coordinates.  When that is this workload's d they are used as
+    they are.  Otherwise the launch is scaled by the rule the counters follow: every
+    algorithmic byte crosses DRAM once, except the part of the optimizer state that the
+    previous launch left in the L2 -- a fixed number of bytes, not a fraction -- so
+    traffic(d) = algorithmic(d) - (algorithmic(d_measured) - measured)."""
     path = os.path.join(ROOT, "profiles", "fused_k8_bf16_dram_traffic.json")
     try:
         with open(path) as f:
             rec = json.load(f)
         if rec.get("kernel_source_hash") != kernel_source_hash():
             return None
-        return float(rec["dram_bytes_per_element"]) * d
+        measured = float(rec["dram_bytes_per_launch"])
+        d_measured = int(rec["d_measured"])
+        if d_measured == d:
+            return measured
+        residue = BYTES_PER_ELEM * d_measured - measured
+        return BYTES_PER_ELEM * d - residue
     except Exception:
         return None
-
-
-class ClockSampler(threading.Thread):
-    """Samples SM clock and clock-event reasons through NVML (read-only) every 20 ms."""
-
-    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
-               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks",
-               0x10: "sync_boost", 0x100: "display_clock"}
-
-    def __init__(self, index):
-        super().__init__(daemon=True)
-        self.index, self.samples, self.stop_flag, self.ok = index, [], False, False
-        self.sm_max = None
-        try:
-            import pynvml
-            self.nv = pynvml
-            pynvml.nvmlInit()
-            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
-            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
-            self.ok = True
-        except Exception:
-            self.ok = False
-
-    def run(self):
-        if not self.ok:
-            return
-        nv = self.nv
-        while not self.stop_flag:
-            try:
-                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
-                try:
-                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
-                except Exception:
-                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
-                try:
-                    watts = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
-                except Exception:
-                    watts = None
-                self.samples.append((time.perf_counter(), mhz, mask, watts))
-            except Exception:
-                pass
-            time.sleep(0.02)
-
-    def summary(self, t0, t1):
-        inside = [s for s in self.samples if t0 <= s[0] <= t1]
-        window = "timed region"
-        if len(inside) < 3:
-            inside, window = list(self.samples), "warm-up + timed region (timed region < 3 samples)"
-        if not inside:
-            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": 0,
-                    "window": "NVML unavailable"}
-        mask = 0
-        for s in inside:
-            mask |= s[2]
-        reasons = sorted(name for bit, name in self.REASONS.items() if mask & bit)
-        watts = [s[3] for s in inside if s[3] is not None]
-        return {"sm_mhz": int(statistics.median(s[1] for s in inside)),
-                "sm_max_mhz": self.sm_max, "reasons": reasons, "samples": len(inside),
-                "power_w_max": max(watts) if watts else None, "window": window}
 
 
 # ------------------------------------------------------------------------- CPU oracle
@@ -223,6 +179,7 @@ def run_ours(args, d):
     import paper_2412_21124_b200 as absnt
     from paper_2412_21124_b200 import dist as adist
     from paper_2412_21124_b200 import synth
+    from paper_2412_21124_b200.clocks import ClockSampler
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -241,32 +198,65 @@ def run_ours(args, d):
     b_next = torch.zeros(1, dtype=torch.int64, device=dev)
     stream = torch.cuda.current_stream()
     launches_per_step = 2  # streaming kernel + finalize kernel
+    step_no = [0]
 
-    def step(i):
-        absnt.abs_normtest_adamw(grads, ETA, B_CUR, stats, None, b_next, p, m, v, HP, STEP0 + i)
+    def step():
+        absnt.abs_normtest_adamw(grads, ETA, B_CUR, stats, None, b_next, p, m, v, HP,
+                                 STEP0 + step_no[0])
+        step_no[0] += 1
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    for i in range(args.warmup):
-        step(i)
+    for _ in range(args.warmup):
+        step()
     torch.cuda.synchronize()
+
+    # The timed region is a sequence of blocks of exactly `steps` back-to-back calls, each
+    # block bracketed by CUDA events on the launching stream, the whole sequence by a barrier
+    # and a synchronize.  One block of a short run (20 steps = 14 ms) is a single sample taken
+    # before the board has reached its steady clocks, so the block is repeated until about a
+    # second of device time has passed, and the reported time is the median block.
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev[0].record(stream)
+    for _ in range(args.steps):
+        step()
+    ev[1].record(stream)
+    torch.cuda.synchronize()
+    est_ms = max(ev[0].elapsed_time(ev[1]), 1e-3)          # a first, untimed block
+    n_blocks = int(min(MAX_BLOCKS, max(MIN_BLOCKS, -(-TIMED_REGION_MS // est_ms))))
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(n_blocks + 1)]
     adist.barrier(dev)
     torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.perf_counter()
-    ev0.record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i)
-    ev1.record(stream)
+    events[0].record(stream)
+    for blk in range(n_blocks):
+        for _ in range(args.steps):
+            step()
+        events[blk + 1].record(stream)
     torch.cuda.synchronize()
     t1 = time.perf_counter()
     adist.barrier(dev)
     torch.cuda.synchronize()
-    sampler.stop_flag = True
-    sampler.join(timeout=2)
-    ms_local = ev0.elapsed_time(ev1) / args.steps
-    ms = adist.max_over_ranks(ms_local, dev)
+    sampler.stop()
+    block_ms_local = [events[i].elapsed_time(events[i + 1]) / args.steps for i in range(n_blocks)]
+    # per block the slowest rank counts; then the median over blocks
+    block_ms = adist.max_over_ranks_vec(block_ms_local, dev)
+    ms = statistics.median(block_ms)
+    ms_local = statistics.median(block_ms_local)
     clocks = sampler.summary(t0, t1)
+    blocks = {"n": n_blocks, "steps_per_block": args.steps, "min_ms": min(block_ms),
+              "median_ms": ms, "max_ms": max(block_ms),
+              "note": "ms per step of each block of `steps` back-to-back calls (max over ranks); "
+                      "ms_per_step is the median block; clocks cover all blocks"}
+    # time x clock per block, where a block is long enough to hold clock samples of its own
+    span = (t1 - t0) / n_blocks
+    per_block_mhz = []
+    for i in range(n_blocks):
+        inside = [s_[1] for s_ in sampler.samples if t0 + i * span <= s_[0] <= t0 + (i + 1) * span]
+        per_block_mhz.append(int(statistics.median(inside)) if len(inside) >= 3 else None)
+    if all(x is not None for x in per_block_mhz):
+        blocks["sm_mhz_per_block"] = per_block_mhz
+        blocks["ms_x_ghz_per_block"] = [t * f / 1e3 for t, f in zip(block_ms, per_block_mhz)]
     final = absnt.read_stats(stats)
     assert final["S"] > 0 and final["n2"] > 0 and int(b_next.item()) >= B_CUR
 
@@ -286,7 +276,7 @@ def run_ours(args, d):
     def e2e_step(i):
         for hg, g in zip(host_grads, grads):
             g.copy_(hg, non_blocking=True)
-        step(i)
+        step()
         host_stats.copy_(stats[:absnt.binding.ABS_STATS_HEADER], non_blocking=True)
         host_b.copy_(b_next, non_blocking=True)
         stream.synchronize()  # the caller needs b_next on the host to resize its sampler
@@ -331,7 +321,8 @@ def run_ours(args, d):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "config": workload_config(d), "clocks": clocks, "e2e": e2e,
-            "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
+            "blocks": blocks,
+            "gpu_launches": launches_per_step * args.steps * n_blocks, "roofline": roofline,
             "cpu_baseline": cpu,
             "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
             "T": final["T"], "b_next": int(b_next.item())}

@@ -93,11 +93,20 @@ __device__ __forceinline__ float2 coord_math_pair(const float2 (&g)[KB], int K,
 //   c = g_0;  S_i = sum_k (g_k - c)^2 - K (gbar - c)^2
 // so that the K values need not all be live at once.  The cancellation is bounded: the
 // first sum exceeds S_i by at most a factor of about K (when g_0 itself is the outlier).
-// K identical values give exactly zero.  The operation order is that of the vector path of
-// chunk_rows_split, so both give identical bits.
+// K identical values give exactly zero.
+// The deviation of the mean, dm = gbar - c, is taken from the unrounded sum and not from the
+// rounded mean: with s = sum_k g_k (exact in fp32 for bf16 inputs within the binade limits,
+// fp64 for fp32 inputs), gbar = fl(s/K) as in the plain form, and dm = fl((s - K c)/K) -- for
+// bf16 one fused multiply-add, whose exact result sum_k (g_k - c) is representable under the
+// same limits; for fp32 one fp64 subtraction.  Were dm formed as fl(gbar) - c, the rounding
+// error delta of gbar would enter S_i to first order (2 K dm delta: relative 2^-24 |mean| /
+// spread, visible once the workers agree to four digits); this way it does not enter at all.
+// The operation order is that of the vector path of chunk_rows_split, so both give identical
+// bits.
 template <typename GT, int KB, bool EXACT, bool WITHQ>
 __device__ __forceinline__ float coord_math_split(const float (&g)[KB], int K,
                                                   const StreamParams& prm, float& dev2, float& sq) {
+  constexpr bool kF32Sum = std::is_same<typename GT::sum_t, float>::value;
   typename GT::sum_t s = 0;
   const float c = g[0];
   float s2 = 0.f;
@@ -110,8 +119,15 @@ __device__ __forceinline__ float coord_math_split(const float (&g)[KB], int K,
       s2 = fmaf(dv, dv, s2);
       if (WITHQ) sq = fmaf(g[k], g[k], sq);
     }
-  const float mean = GT::template mean<false>(s, prm);
-  const float dm = mean - c;
+  float mean, dm;
+  if constexpr (kF32Sum) {
+    mean = mean_of_sum<false>(s, prm.inv_Kf, prm.neg_Kf);
+    dm = fmaf(prm.neg_Kf, c, s) * prm.inv_Kf;
+  } else {
+    const double mx = s * prm.inv_K;
+    mean = static_cast<float>(mx);
+    dm = static_cast<float>(mx - static_cast<double>(c));
+  }
   dev2 = clamp_nonneg(fmaf(prm.neg_Kf * dm, dm, s2));
   return mean;
 }
@@ -467,13 +483,13 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
               c[pi] = g;
               neg_c[pi] = make_float2(-g.x, -g.y);
             }
+            const float2 dv = __fadd2_rn(g, neg_c[pi]);
             if constexpr (kF32Sum) {
               sp[pi] = __fadd2_rn(sp[pi], g);
             } else {
               s[2 * pi] += static_cast<typename GT::sum_t>(g.x);
               s[2 * pi + 1] += static_cast<typename GT::sum_t>(g.y);
             }
-            const float2 dv = __fadd2_rn(g, neg_c[pi]);
             s2[pi] = __ffma2_rn(dv, dv, s2[pi]);
             if (WITHQ) q[pi] = __ffma2_rn(g, g, q[pi]);
           }
@@ -509,13 +525,17 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
       float2* v2 = reinterpret_cast<float2*>(&pv);
 #pragma unroll
       for (int pi = 0; pi < P; ++pi) {
-        float2 mean;
-        if constexpr (kF32Sum)
+        float2 mean, dm;
+        if constexpr (kF32Sum) {
           mean = mean_of_sum2<false>(sp[pi], prm.inv_Kf, prm.neg_Kf);
-        else
-          mean = make_float2(GT::template mean<false>(s[2 * pi], prm),
-                             GT::template mean<false>(s[2 * pi + 1], prm));
-        const float2 dm = __fadd2_rn(mean, neg_c[pi]);
+          dm = __fmul2_rn(__ffma2_rn(make_float2(prm.neg_Kf, prm.neg_Kf), c[pi], sp[pi]),
+                          make_float2(prm.inv_Kf, prm.inv_Kf));
+        } else {
+          const double mx = s[2 * pi] * prm.inv_K, my = s[2 * pi + 1] * prm.inv_K;
+          mean = make_float2(static_cast<float>(mx), static_cast<float>(my));
+          dm = make_float2(static_cast<float>(mx - static_cast<double>(c[pi].x)),
+                           static_cast<float>(my - static_cast<double>(c[pi].y)));
+        }
         const float2 t = __ffma2_rn(__fmul2_rn(make_float2(prm.neg_Kf, prm.neg_Kf), dm), dm, s2[pi]);
         gb[2 * pi] = mean.x;
         gb[2 * pi + 1] = mean.y;

@@ -110,6 +110,14 @@ def max_over_ranks(x, device="cpu"):
     return float(t.item())
 
 
+def max_over_ranks_vec(xs, device="cpu"):
+    """Element-wise max over ranks of a list of floats (one all-reduce)."""
+    t = torch.tensor([float(x) for x in xs], dtype=torch.float64, device=device)
+    if dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 def sum_over_ranks(x, device="cpu"):
     t = torch.tensor([float(x)], dtype=torch.float64, device=device)
     if dist.is_initialized() and dist.get_world_size() > 1:

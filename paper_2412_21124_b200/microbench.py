@@ -2,6 +2,11 @@
 
   python -m paper_2412_21124_b200.microbench --call fused --d 33554432 --K 8 --dtype bf16
   python -m paper_2412_21124_b200.microbench --sweep            # the d x K x dtype grid
+  python -m paper_2412_21124_b200.microbench --report           # the grid and every other call
+  python -m paper_2412_21124_b200.microbench --format out.jsonl # those lines as markdown tables
+
+Every point carries the SM clock (median over the timed region), the clock-event reasons seen
+and the peak power draw, read through NVML while the point was timed.
 
 Timing: CUDA events on the launching stream around `steps` back-to-back calls after
 `warmup` calls; calls whose first estimate is under ~200 us (where the host's per-call cost of
@@ -13,12 +18,15 @@ adamw 28 (+2 with --mixed), persample 4 per matrix element.
 """
 import argparse
 import json
+import os
 import sys
+import time
 
 import torch
 
 from . import binding as B
 from . import synth
+from .clocks import ClockSampler
 
 HP = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
 L2_BYTES = 126 * 1024 * 1024
@@ -110,6 +118,9 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
     if graph is None:  # short calls are bound by the host's per-call cost, which the estimate includes
         graph = est_ms is not None and est_ms < 0.2
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    t_begin = None
     if graph:
         # capture the calls once, replay them: device-side time of back-to-back calls
         per_graph = max(n_sets, min(steps, 64))
@@ -124,6 +135,10 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
         replays = max(1, steps // per_graph)
         g.replay()
         torch.cuda.synchronize()
+        # short calls: replay for at least ~150 ms so that the clock record has samples
+        per_replay_ms = max(est_ms if est_ms is not None else 0.05, 1e-3) * per_graph
+        replays = int(max(replays, min(2000, 150.0 / per_replay_ms)))
+        t_begin = time.perf_counter()
         e0.record()
         for _ in range(replays):
             g.replay()
@@ -132,11 +147,14 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
         steps = replays * per_graph
     else:
         stream = torch.cuda.current_stream()
+        t_begin = time.perf_counter()
         e0.record(stream)
         for i in range(steps):
             one(warmup + i)
         e1.record(stream)
         torch.cuda.synchronize()
+    t_end = time.perf_counter()
+    sampler.stop()
     ms = e0.elapsed_time(e1) / steps
     out = {"call": call, "d": d, "K": K, "dtype": dtype, "n_shards": n_shards, "gbar": bool(gbar),
            "mixed": bool(mixed), "steps": steps, "buffer_sets": n_sets, "cuda_graph": bool(graph),
@@ -144,7 +162,104 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
            "bytes": nbytes, "GBps": nbytes / (ms * 1e-3) / 1e9}
     if call == "persample":
         out["b"] = b
+    ck = sampler.summary(t_begin, t_end)
+    out["clocks"] = {"sm_mhz": ck["sm_mhz"], "sm_max_mhz": ck["sm_max_mhz"],
+                     "reasons": ck["reasons"], "power_w_max": ck.get("power_w_max"),
+                     "samples": ck["samples"], "window": ck["window"]}
     return out
+
+
+# Every per-call number quoted beside the d x K grid, as (call, d, K, dtype, shards, extras).
+GPT2, LLAMA = 124_439_808, 1_235_814_400
+REPORT_POINTS = (
+    [("normtest", LLAMA, 8, "bf16", 8, {})]
+    + [("normtest", GPT2, K, dt, 1, {}) for K in (1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14,
+                                                  15, 16, 24, 32) for dt in ("bf16", "f32")]
+    + [("adamw", GPT2, 0, "f32", 1, {}), ("adamw", LLAMA, 0, "f32", 1, {}),
+       ("adamw", GPT2, 0, "f32", 1, {"mixed": True})]
+    + [("persample", 16_384, 0, "f32", 1, {"b": b}) for b in (4096, 1024, 256, 32)]
+    + [("persample", 65_536, 0, "f32", 1, {"b": 4096})]
+    + [("fused", GPT2, 8, "bf16", 1, {"gbar": True}), ("fused", GPT2, 8, "bf16", 1, {"mixed": True}),
+       ("fused", 1_048_576, 4, "f32", 1, {})]
+    + [("fused", GPT2, K, "bf16", 1, {}) for K in (6, 12, 20, 24, 27, 31, 36, 40, 44, 48, 52, 56,
+                                                   60, 64)]
+    + [("fused", GPT2, K, "f32", 1, {}) for K in (12, 20, 31, 48, 64)]
+    # the paper's own model sizes (Table 4), J = 4 workers, bf16
+    + [("fused", d, 4, "bf16", 1, {}) for d in (304_600_000, 1_100_000_000, 3_400_000_000)])
+
+
+def sweep(args, graph):
+    for dtype in ("bf16", "f32"):
+        esz = 2 if dtype == "bf16" else 4
+        for d in SWEEP_D:
+            for K in SWEEP_K:
+                if K * d * esz + 16 * d > MEM_CAP:
+                    print(json.dumps({"call": "fused", "d": d, "K": K, "dtype": dtype, "sweep": True,
+                                      "skipped": "K*d*s + 16*d exceeds 160 GB"}), flush=True)
+                    continue
+                r = run_point("fused", d, K, dtype, steps=args.steps, warmup=args.warmup, graph=graph)
+                r["sweep"] = True
+                print(json.dumps(r), flush=True)
+                torch.cuda.empty_cache()
+
+
+def report(args, graph):
+    sweep(args, graph)
+    for call, d, K, dtype, shards, extra in REPORT_POINTS:
+        r = run_point(call, d, K, dtype, shards, args.steps, args.warmup, extra.get("gbar", False),
+                      extra.get("b", 4096), graph=graph, mixed=extra.get("mixed", False))
+        print(json.dumps(r), flush=True)
+        torch.cuda.empty_cache()
+
+
+def _measured_peak():
+    here = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    try:
+        with open(os.path.join(here, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"])
+    except Exception:
+        return None
+
+
+def format_markdown(path):
+    """The JSON lines of --sweep / --report as two markdown tables (stdout)."""
+    rows = [json.loads(line) for line in open(path) if line.startswith("{")]
+    peak = _measured_peak()
+
+    def clk(r):
+        c = r.get("clocks") or {}
+        if c.get("sm_mhz") is None:
+            return "-", "-"
+        watts = "%.0f W" % c["power_w_max"] if c.get("power_w_max") else ""
+        return "%d" % c["sm_mhz"], (",".join(c.get("reasons") or []) or "none") + " " + watts
+
+    print("| dtype | d | K | ms | GB/s | of 8000 | of measured | steps | graph | SM MHz | reasons, peak power |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        if not r.get("sweep"):
+            continue
+        if "skipped" in r:
+            print("| %s | %d | %d | skipped: %s | | | | | | | |" % (r["dtype"], r["d"], r["K"],
+                                                                  r["skipped"]))
+            continue
+        mhz, why = clk(r)
+        print("| %s | %d | %d | %.4f | %.0f | %.3f | %s | %d | %s | %s | %s |" % (
+            r["dtype"], r["d"], r["K"], r["ms"], r["GBps"], r["GBps"] / 8000.0,
+            "%.3f" % (r["GBps"] / peak) if peak else "-", r["steps"],
+            "yes" if r["cuda_graph"] else "", mhz, why))
+    print()
+    print("| call | d | K / b | dtype | shards | ms | GB/s | of 8000 | graph | SM MHz | reasons, peak power |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        if r.get("sweep"):
+            continue
+        name = r["call"] + (" +gbar" if r.get("gbar") and r["call"] == "fused" else "") + (
+            " +bf16 copy" if r.get("mixed") else "")
+        kb = r["b"] if r["call"] == "persample" else (r["K"] if r["call"] != "adamw" else "-")
+        mhz, why = clk(r)
+        print("| %s | %d | %s | %s | %d | %.4f | %.0f | %.3f | %s | %s | %s |" % (
+            name, r["d"], kb, r["dtype"], r["n_shards"], r["ms"], r["GBps"], r["GBps"] / 8000.0,
+            "yes" if r["cuda_graph"] else "", mhz, why))
 
 
 def main(argv=None):
@@ -161,29 +276,28 @@ def main(argv=None):
     ap.add_argument("--mixed", action="store_true",
                     help="fused / adamw: also write the bf16 copy of the parameters")
     ap.add_argument("--sweep", action="store_true", help="fused call over the d x K x dtype grid")
+    ap.add_argument("--report", action="store_true",
+                    help="the grid and the per-call points quoted beside it, in one run")
+    ap.add_argument("--format", metavar="JSONL", default=None,
+                    help="print the JSON lines of a --sweep/--report run as markdown tables")
     ap.add_argument("--graph", choices=["auto", "on", "off"], default="auto",
                     help="time replays of a captured CUDA graph (auto: for calls under 200 us)")
     args = ap.parse_args(argv)
+    if args.format:
+        format_markdown(args.format)
+        return
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device (there is no CPU fallback)")
     B.lib()
     graph = {"auto": None, "on": True, "off": False}[args.graph]
-    if not args.sweep:
+    if args.report:
+        report(args, graph)
+    elif args.sweep:
+        sweep(args, graph)
+    else:
         print(json.dumps(run_point(args.call, args.d, args.K, args.dtype, args.shards, args.steps,
                                    args.warmup, args.gbar, args.b, graph=graph,
                                    mixed=args.mixed)), flush=True)
-        return
-    for dtype in ("bf16", "f32"):
-        esz = 2 if dtype == "bf16" else 4
-        for d in SWEEP_D:
-            for K in SWEEP_K:
-                if K * d * esz + 16 * d > MEM_CAP:
-                    print(json.dumps({"call": "fused", "d": d, "K": K, "dtype": dtype,
-                                      "skipped": "K*d*s + 16*d exceeds 160 GB"}), flush=True)
-                    continue
-                r = run_point("fused", d, K, dtype, steps=args.steps, warmup=args.warmup, graph=graph)
-                print(json.dumps(r), flush=True)
-                torch.cuda.empty_cache()
 
 
 if __name__ == "__main__":
