@@ -28,6 +28,11 @@
  *   abs_oracle_persample   the approximate norm test on per-sample gradients
  *                          (Eq. 3 with the Var definition displayed after Eq. 2, and
  *                          the b_{k+1} display after Eq. 3).
+ *   abs_oracle_norm_test_coordwise / abs_oracle_persample_coordwise
+ *                          the coordinate-wise norm test (Sec. 4, the test Proposition 1 and
+ *                          Theorem 1 are stated for; Appendix B, first remark, prints it for
+ *                          the exact variance).  The paper gives no sample form; the reading
+ *                          is stated above the function.
  *   abs_oracle_adamw       the AdamW lines of Algorithm 1.
  *   abs_oracle_round_batch the three rounding lines of Algorithm 1's If branch.
  *   abs_oracle_bf16_round  the bfloat16 working copy of fp32 parameters (Sec. 5: bfloat16
@@ -258,6 +263,156 @@ int abs_oracle_persample(const void* G, int64_t b, int64_t d, int64_t ld, int dt
   totals[TOT_FLAGS] = (double)flags;
   totals[TOT_NORM] = (double)(b - 1);
   return 0;
+}
+
+/*
+ * Coordinate-wise norm test (Sec. 4; Appendix B, first remark).  The paper states it for the
+ * exact variance only: for every coordinate i,
+ *     E_k[(d_i L_B(w_k) - d_i L(w_k))^2] <= eta^2 (d_i L(w_k))^2,
+ * and says its experiments use the summed test instead.  Reading (the sample form, built the
+ * way Eq. 5 is built from the exact-variance test, Eq. 4): the variance of coordinate i of the
+ * batch gradient is estimated by [\hat Var]_i / b, coordinate i of the estimator displayed
+ * before Eq. 5, and d_i L by gbar_i:
+ *     [\hat Var]_i / b <= eta^2 gbar_i^2      for every i,    [\hat Var]_i = (1/norm) sum_k (g_k[i]-gbar_i)^2
+ * Per coordinate T_i = [\hat Var]_i / (eta^2 gbar_i^2); the test holds iff T = max_i T_i <= b,
+ * and as in the display after Eq. 3 the next batch size is the smallest one under which, by the
+ * same heuristic, every coordinate would pass: b_next = ceil(T) if T > b else b.
+ *   [\hat Var]_i = 0          T_i = 0 (the coordinate passes for any b, also when gbar_i = 0)
+ *   [\hat Var]_i > 0, gbar_i = 0   T_i = +inf
+ * argmax = the smallest i that attains the maximum.  Flags: NONFINITE (and T = NaN, b kept)
+ * when n2 or S is not finite; else DEGENERATE when n2 = 0 or T = +inf; VIOLATED when T > b.
+ * The summed statistic of the same data is (S/norm)/(eta^2 n2), a weighted mean of the T_i
+ * with weights gbar_i^2, so T >= it always.
+ */
+typedef struct {
+  double n2, S, Q, tmax;
+  int64_t arg;
+} cw_run;
+
+/* the statistic of one coordinate from its K (or b) values, read with stride `stride` */
+static double cw_coordinate(const void* const* grads, const void* G, int64_t stride, int n,
+                            int dtype, int64_t i, double norm, double eta, double* gbar_i,
+                            double* dev2_i, double* q_i) {
+  double sum = 0.0;
+  for (int k = 0; k < n; ++k)
+    sum += grads ? widen(grads[k], dtype, i) : widen(G, dtype, (int64_t)k * stride + i);
+  const double gbar = sum / (double)n;
+  double dev2 = 0.0, q = 0.0;
+  for (int k = 0; k < n; ++k) {
+    const double g = grads ? widen(grads[k], dtype, i) : widen(G, dtype, (int64_t)k * stride + i);
+    dev2 += (g - gbar) * (g - gbar);
+    q += g * g;
+  }
+  *gbar_i = gbar;
+  *dev2_i = dev2;
+  *q_i = q;
+  if (dev2 == 0.0) return 0.0;
+  return (dev2 / norm) / ((eta * eta) * (gbar * gbar)); /* +inf when gbar == 0 */
+}
+
+static int cw_test(const void* const* grads, const void* G, int64_t stride, int n, int64_t d,
+                   int dtype, const int64_t* shard_offsets, int n_shards, double norm, double eta,
+                   int64_t b_cur, double* gbar_out, double* ratio_out, double* totals,
+                   double* shard_max, int64_t* argmax_out, int64_t* b_next_out) {
+  int64_t one_shard[2] = {0, d};
+  if (!shard_offsets) {
+    shard_offsets = one_shard;
+    n_shards = 1;
+  }
+  if (n_shards < 1 || shard_offsets[0] != 0 || shard_offsets[n_shards] != d) return -1;
+  double n2 = 0.0, S = 0.0, Q = 0.0, tmax = 0.0;
+  int64_t arg = 0;
+  for (int s = 0; s < n_shards; ++s) {
+    const int64_t lo = shard_offsets[s], hi = shard_offsets[s + 1];
+    if (hi < lo) return -1;
+    const int64_t n_runs = (hi - lo + ABS_ORACLE_CHUNK - 1) / ABS_ORACLE_CHUNK;
+    cw_run* run = (cw_run*)malloc((size_t)(n_runs > 0 ? n_runs : 1) * sizeof(cw_run));
+    if (!run) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < n_runs; ++r) {
+      const int64_t i0 = lo + r * ABS_ORACLE_CHUNK;
+      const int64_t i1 = (i0 + ABS_ORACLE_CHUNK < hi) ? i0 + ABS_ORACLE_CHUNK : hi;
+      cw_run a = {0.0, 0.0, 0.0, -1.0, i0};
+      for (int64_t i = i0; i < i1; ++i) {
+        double gbar, dev2, q;
+        const double t = cw_coordinate(grads, G, stride, n, dtype, i, norm, eta, &gbar, &dev2, &q);
+        if (gbar_out) gbar_out[i] = gbar;
+        if (ratio_out) ratio_out[i] = t;
+        a.n2 += gbar * gbar;
+        a.S += dev2;
+        a.Q += q;
+        if (t > a.tmax) { /* strict: the first index keeps a tie; NaN never wins */
+          a.tmax = t;
+          a.arg = i;
+        }
+      }
+      run[r] = a;
+    }
+    double sn2 = 0.0, sS = 0.0, sQ = 0.0, smax = -1.0;
+    int64_t sarg = lo;
+    for (int64_t r = 0; r < n_runs; ++r) {
+      sn2 += run[r].n2;
+      sS += run[r].S;
+      sQ += run[r].Q;
+      if (run[r].tmax > smax) {
+        smax = run[r].tmax;
+        sarg = run[r].arg;
+      }
+    }
+    free(run);
+    if (smax < 0.0) smax = 0.0; /* an empty shard, or one whose ratios are all NaN */
+    if (shard_max) shard_max[s] = smax;
+    n2 += sn2;
+    S += sS;
+    Q += sQ;
+    if (smax > tmax) {
+      tmax = smax;
+      arg = sarg;
+    }
+  }
+  int flags = 0;
+  double T = tmax;
+  int64_t b_next = b_cur;
+  if (!isfinite(S) || !isfinite(n2)) {
+    flags |= ABS_ORACLE_FLAG_NONFINITE;
+    T = NAN;
+  } else {
+    if (n2 == 0.0 || isinf(T)) flags |= ABS_ORACLE_FLAG_DEGENERATE;
+    if (T > (double)b_cur) {
+      flags |= ABS_ORACLE_FLAG_VIOLATED;
+      b_next = (T >= 4611686018427387904.0) ? INT64_MAX : (int64_t)ceil(T);
+    }
+  }
+  memset(totals, 0, TOT_COUNT * sizeof(double));
+  totals[TOT_N2] = n2;
+  totals[TOT_S] = S;
+  totals[TOT_Q] = Q;
+  totals[TOT_T] = T;
+  totals[TOT_FLAGS] = (double)flags;
+  totals[TOT_NORM] = norm;
+  if (argmax_out) *argmax_out = arg;
+  *b_next_out = b_next;
+  return 0;
+}
+
+/* worker form: norm = K (the estimator carries 1/J) */
+int abs_oracle_norm_test_coordwise(const void* const* grads, int K, int64_t d, int dtype,
+                                   const int64_t* shard_offsets, int n_shards, double eta,
+                                   int64_t b_cur, double* gbar_out, double* ratio_out,
+                                   double* totals, double* shard_max, int64_t* argmax_out,
+                                   int64_t* b_next_out) {
+  if (!grads || K < 1 || d < 1 || !totals || !b_next_out) return -1;
+  return cw_test(grads, NULL, 0, K, d, dtype, shard_offsets, n_shards, (double)K, eta, b_cur,
+                 gbar_out, ratio_out, totals, shard_max, argmax_out, b_next_out);
+}
+
+/* per-sample form: rows of G are the samples, norm = b-1 (the Var display after Eq. 2) */
+int abs_oracle_persample_coordwise(const void* G, int64_t b, int64_t d, int64_t ld, int dtype,
+                                   double eta, double* gbar_out, double* ratio_out,
+                                   double* totals, int64_t* argmax_out, int64_t* b_next_out) {
+  if (!G || b < 2 || b > INT32_MAX || d < 1 || ld < d || !totals || !b_next_out) return -1;
+  return cw_test(NULL, G, ld, (int)b, d, dtype, NULL, 1, (double)(b - 1), eta, b, gbar_out,
+                 ratio_out, totals, NULL, argmax_out, b_next_out);
 }
 
 /*

@@ -51,6 +51,12 @@ def lib():
                                            ptr, ptr]
         L.abs_oracle_persample.restype = cint
         L.abs_oracle_persample.argtypes = [ptr, i64, i64, i64, cint, dbl, ptr, ptr, ptr]
+        L.abs_oracle_norm_test_coordwise.restype = cint
+        L.abs_oracle_norm_test_coordwise.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64,
+                                                     ptr, ptr, ptr, ptr, ptr, ptr]
+        L.abs_oracle_persample_coordwise.restype = cint
+        L.abs_oracle_persample_coordwise.argtypes = [ptr, i64, i64, i64, cint, dbl, ptr, ptr, ptr,
+                                                     ptr, ptr]
         L.abs_oracle_adamw.restype = cint
         L.abs_oracle_adamw.argtypes = [ptr, ptr, ptr, ptr, i64, dbl, dbl, dbl, dbl, dbl, i64,
                                        ptr, ptr, ptr]
@@ -130,6 +136,57 @@ def persample(G, eta, want_gbar=True):
         raise ValueError("abs_oracle_persample rejected its arguments")
     out = _totals_dict(tot, b_next.value)
     out["gbar"] = gbar
+    return out
+
+
+def norm_test_coordwise(grads, eta, b_cur, shard_offsets=None, want_ratios=False):
+    """Coordinate-wise test, worker form.  Returns the dict of norm_test (T, flags and b_next
+    are those of the coordinate-wise test) plus "argmax", "shard_max" and, on request,
+    "ratios" (the d per-coordinate statistics T_i)."""
+    grads = [np.ascontiguousarray(g) for g in grads]
+    K, d = len(grads), int(grads[0].shape[0])
+    code = _dtype_code(grads[0])
+    for g in grads:
+        assert g.ndim == 1 and g.shape[0] == d and _dtype_code(g) == code
+    ptrs = (ctypes.c_void_p * K)(*[g.ctypes.data for g in grads])
+    if shard_offsets is None:
+        n_shards, offs_p = 1, None
+    else:
+        offs = np.ascontiguousarray(np.asarray(shard_offsets, dtype=np.int64))
+        n_shards, offs_p = int(offs.shape[0]) - 1, _p(offs)
+    gbar = np.empty(d, dtype=np.float64)
+    ratios = np.empty(d, dtype=np.float64) if want_ratios else None
+    tot = np.zeros(TOT_COUNT, dtype=np.float64)
+    shard_max = np.zeros(n_shards, dtype=np.float64)
+    b_next, arg = ctypes.c_int64(0), ctypes.c_int64(0)
+    rc = lib().abs_oracle_norm_test_coordwise(ptrs, K, d, code, offs_p, n_shards, float(eta),
+                                              int(b_cur), _p(gbar),
+                                              _p(ratios) if want_ratios else None, _p(tot),
+                                              _p(shard_max), ctypes.byref(arg),
+                                              ctypes.byref(b_next))
+    if rc != 0:
+        raise ValueError("abs_oracle_norm_test_coordwise rejected its arguments")
+    out = _totals_dict(tot, b_next.value)
+    out.update(gbar=gbar, ratios=ratios, argmax=int(arg.value), shard_max=shard_max)
+    return out
+
+
+def persample_coordwise(G, eta, want_ratios=False):
+    """Coordinate-wise test, per-sample form (rows of G are the samples)."""
+    assert G.ndim == 2 and G.strides[1] == G.itemsize and G.strides[0] % G.itemsize == 0
+    b, d = int(G.shape[0]), int(G.shape[1])
+    ld = G.strides[0] // G.itemsize
+    gbar = np.empty(d, dtype=np.float64)
+    ratios = np.empty(d, dtype=np.float64) if want_ratios else None
+    tot = np.zeros(TOT_COUNT, dtype=np.float64)
+    b_next, arg = ctypes.c_int64(0), ctypes.c_int64(0)
+    rc = lib().abs_oracle_persample_coordwise(_p(G), b, d, ld, _dtype_code(G), float(eta),
+                                              _p(gbar), _p(ratios) if want_ratios else None,
+                                              _p(tot), ctypes.byref(arg), ctypes.byref(b_next))
+    if rc != 0:
+        raise ValueError("abs_oracle_persample_coordwise rejected its arguments")
+    out = _totals_dict(tot, b_next.value)
+    out.update(gbar=gbar, ratios=ratios, argmax=int(arg.value))
     return out
 
 

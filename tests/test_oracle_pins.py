@@ -487,6 +487,139 @@ def test_bf16_round_against_torch_and_hand_cases():
     assert (nan & 0x7F80) == 0x7F80 and (nan & 0x007F) != 0
 
 
+# --------------------------------------------------------------- coordinate-wise test
+def frac_coordwise(rows, norm, eta):
+    """Exact per-coordinate statistics T_i (Fractions; None stands for +inf)."""
+    K, d = len(rows), len(rows[0])
+    F = [[Fraction(float(x)) for x in r] for r in rows]
+    e2 = Fraction(float(eta)) ** 2
+    out = []
+    for i in range(d):
+        gbar = sum(F[k][i] for k in range(K)) / K
+        var = sum((F[k][i] - gbar) ** 2 for k in range(K)) / norm
+        if var == 0:
+            out.append(Fraction(0))
+        elif gbar == 0:
+            out.append(None)
+        else:
+            out.append(var / (e2 * gbar * gbar))
+    return out
+
+
+def test_hand_cases_coordwise():
+    cases = json.load(open(GOLDEN))["coordwise"]
+    c = cases[0]
+    grads = [np.asarray(g, dtype=np.float32) for g in c["grads"]]
+    for dec in c["decisions"]:
+        r = orc.norm_test_coordwise(grads, c["eta"], dec["b_cur"], want_ratios=True)
+        assert list(r["ratios"]) == c["ratios"] and r["T"] == c["T"] and r["argmax"] == c["argmax"]
+        assert r["b_next"] == dec["b_next"]
+        assert bool(r["flags"] & orc.FLAG_VIOLATED) == dec["violated"]
+        # the summed test on the same data decides differently at b = 2
+        s = orc.norm_test(grads, c["eta"], dec["b_cur"])
+        assert Fraction(s["T"]).limit_denominator(1000) == Fraction(*c["T_sum_fraction"])
+        assert s["b_next"] == dec["b_next_summed"]
+    r = orc.persample_coordwise(np.stack(grads), c["eta"])
+    assert r["T"] == c["T_persample"] and r["b_next"] == c["b_next_persample"]
+    c = cases[1]
+    grads = [np.asarray(g, dtype=np.float32) for g in c["grads"]]
+    r = orc.norm_test_coordwise(grads, c["eta"], 7, want_ratios=True)
+    assert [("inf" if math.isinf(x) else x) for x in r["ratios"]] == c["ratios"]
+    assert r["T"] == math.inf and r["argmax"] == c["argmax"] and r["flags"] == c["flags"]
+    assert r["b_next"] == 2 ** 63 - 1
+    r = orc.norm_test_coordwise([g[1:] for g in grads], c["eta"], 7)
+    assert r["T"] == 0.0 and r["flags"] == 0 and r["b_next"] == 7
+    z = [np.zeros(3, dtype=np.float32)] * 2
+    r = orc.norm_test_coordwise(z, c["eta"], 7)
+    assert r["T"] == 0.0 and r["flags"] == orc.FLAG_DEGENERATE and r["b_next"] == 7
+
+
+@pytest.mark.parametrize("K,d", [(1, 1), (2, 3), (3, 5), (4, 8), (5, 7), (7, 2)])
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+def test_coordwise_brute_force_rational(K, d, kind):
+    rng = np.random.default_rng(300 + 10 * K + d)
+    raw = rng.normal(0.1, 1.0, size=(K, d)).astype(np.float32)
+    raw[:, 0] = raw[0, 0]                      # a zero-variance coordinate
+    if kind == "bf16":
+        bits = [bf16_bits(r) for r in raw]
+        vals = [bf16_to_f64(b) for b in bits]
+        grads = bits
+    else:
+        vals = [r.astype(np.float64) for r in raw]
+        grads = [r for r in raw]
+    eta = 0.375
+    want = frac_coordwise([list(v) for v in vals], K, eta)
+    finite = [w for w in want if w is not None]
+    T = max(finite)
+    arg = want.index(T)
+    for b_cur in (1, 3, 10 ** 6):
+        r = orc.norm_test_coordwise(grads, eta, b_cur, want_ratios=True)
+        for got, w in zip(r["ratios"], want):
+            assert got == pytest.approx(float(w), rel=1e-13)
+        assert r["ratios"][0] == 0.0
+        assert r["T"] == pytest.approx(float(T), rel=1e-13) and r["argmax"] == arg
+        assert r["b_next"] == (math.ceil(T) if T > b_cur else b_cur)
+    # per-sample form: the rows are the samples, normalisation b-1
+    if K >= 2 and kind == "f32":
+        want = frac_coordwise([list(v) for v in vals], K - 1, eta)
+        r = orc.persample_coordwise(raw, eta, want_ratios=True)
+        for got, w in zip(r["ratios"], want):
+            assert got == pytest.approx(float(w), rel=1e-13)
+        T = max(want)
+        assert r["b_next"] == (math.ceil(T) if T > K else K) and r["argmax"] == want.index(T)
+
+
+def test_coordwise_against_numpy_and_invariants():
+    rng = np.random.default_rng(31)
+    K, d, eta = 8, 12_345, 0.2
+    grads = [rng.normal(0.05, 0.3, size=d).astype(np.float32) for _ in range(K)]
+    G = np.stack(grads).astype(np.float64)
+    t = G.var(axis=0, ddof=0) / (eta ** 2 * G.mean(axis=0) ** 2)
+    offs = [0, 100, 100, 5000, d]
+    r = orc.norm_test_coordwise(grads, eta, 64, shard_offsets=offs, want_ratios=True)
+    np.testing.assert_allclose(r["ratios"], t, rtol=1e-11)
+    assert r["argmax"] == int(np.argmax(t)) and r["T"] == pytest.approx(t.max(), rel=1e-11)
+    # shard maxima: the maximum over the shard's slice; an empty shard reports 0
+    for s in range(4):
+        want = t[offs[s]:offs[s + 1]].max() if offs[s + 1] > offs[s] else 0.0
+        assert r["shard_max"][s] == pytest.approx(want, rel=1e-11)
+    assert r["T"] == r["shard_max"].max()
+    # the sums are those of the summed test, and the coordinate-wise statistic dominates the
+    # summed one (which is a weighted mean of the T_i with weights gbar_i^2)
+    s = orc.norm_test(grads, eta, 64, shard_offsets=offs)
+    for key in ("n2", "S", "Q"):   # same sums, another order of additions
+        assert r[key] == pytest.approx(s[key], rel=1e-12)
+    assert r["T"] >= s["T"]
+    # one coordinate: the two statistics are the same expression
+    one = [g[7:8] for g in grads]
+    assert orc.norm_test_coordwise(one, eta, 64)["T"] == orc.norm_test(one, eta, 64)["T"]
+    # scaling every gradient by a power of two changes no ratio; a permutation of the
+    # coordinates moves the argmax with it
+    r2 = orc.norm_test_coordwise([4.0 * g for g in grads], eta, 64, want_ratios=True)
+    assert np.array_equal(r2["ratios"], r["ratios"])
+    perm = rng.permutation(d)
+    r3 = orc.norm_test_coordwise([g[perm] for g in grads], eta, 64)
+    assert r3["T"] == r["T"] and perm[r3["argmax"]] == r["argmax"]
+    # T scales with 1/eta^2, so b_next never grows with eta
+    seen = [orc.norm_test_coordwise(grads, e, 64)["b_next"] for e in (0.05, 0.1, 0.2, 0.4, 3.0, 1e4)]
+    assert seen == sorted(seen, reverse=True) and seen[-1] == 64
+    # per-sample form against numpy's ddof=1
+    Gs = rng.normal(0.02, 0.3, size=(33, 700)).astype(np.float32)
+    tp = Gs.astype(np.float64).var(axis=0, ddof=1) / (eta ** 2 * Gs.astype(np.float64).mean(axis=0) ** 2)
+    rp = orc.persample_coordwise(Gs, eta, want_ratios=True)
+    np.testing.assert_allclose(rp["ratios"], tp, rtol=1e-11)
+    assert rp["argmax"] == int(np.argmax(tp)) and rp["norm"] == 32
+    # a strided matrix is read row by row, not transposed
+    wide = np.zeros((33, 704), dtype=np.float32)
+    wide[:, :700] = Gs
+    assert orc.persample_coordwise(wide[:, :700], eta)["T"] == rp["T"]
+    # non-finite input: flag, T = NaN, batch size kept
+    bad = [g.copy() for g in grads]
+    bad[3][17] = np.nan
+    rb = orc.norm_test_coordwise(bad, eta, 64)
+    assert rb["flags"] == orc.FLAG_NONFINITE and math.isnan(rb["T"]) and rb["b_next"] == 64
+
+
 def test_thread_count_does_not_change_results():
     code = (
         "import sys, numpy as np; sys.path.insert(0, %r)\n"
