@@ -82,6 +82,7 @@ enum {
   ABS_STAT_FLAGS = 4,   /* ABS_FLAG_* bits stored as a double                            */
   ABS_STAT_NORM = 5,    /* K (worker form) or b-1 (per-sample form)                      */
   ABS_STAT_NCHUNKS = 6, /* number of reduction chunks the call used                      */
+  ABS_STAT_ARGMAX = 7,  /* coordinate-wise calls: the coordinate with the largest T_i; else 0 */
   ABS_STATS_HEADER = 8
 };
 /* then n_shards records of ABS_SHARD_STRIDE doubles {n2_s, S_s, Q_s, 0}, in shard order,
@@ -107,7 +108,7 @@ size_t abs_persample_stats_bytes(int64_t b, int64_t d);
  * DDP-Norm / FSDP-Norm test (Sec. 3.2-3.3; Algorithm 1 from "Compute the batch
  * gradient" through the If/Else on T_k).
  *   gbar[i] = (1/K) sum_k g_k[i]                      (mean over workers, fp32 out)
- *   n2 = sum_i gbar[i]^2,  S = sum_k sum_i (g_k[i]-gbar[i])^2,  Q = sum_k sum_i g_k[i]^2
+ *   n2 = sum_i gbar[i]^2,  S = sum_k sum_i (g_k[i]-gbar[i])^2
  *   T = (S/K) / (eta^2 n2);   b_next = ceil(T) if T > b_cur else b_cur
  * The same sums are also reported per shard of the flat vector (FSDP-Norm: each
  * worker holds one parameter shard; Appendix A concatenates them); the totals are
@@ -126,10 +127,18 @@ size_t abs_persample_stats_bytes(int64_t b, int64_t d);
  *   gbar_out       device, d floats; must not overlap any grads[k] (ABS_ERR_ALIAS)
  *   b_next_out     device, one int64
  * Non-finite inputs are not an error: the flag is raised and b_next = b_cur.
+ * The diagnostic Q is not computed (its slots read NaN): no decision uses it and it costs the
+ * test, which is bound by instruction issue, 1-6% of its bandwidth.
  */
 int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                   const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
                   void* stats_out, float* gbar_out, int64_t* b_next_out, abs_stream_t stream);
+
+/* abs_norm_test that also accumulates the diagnostic Q = sum_k sum_i g_k[i]^2, per shard and
+ * in total (the identity S = Q - K*n2 checks a run's sums against each other). */
+int abs_norm_test_q(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                    const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                    void* stats_out, float* gbar_out, int64_t* b_next_out, abs_stream_t stream);
 
 /*
  * AdamW update (Algorithm 1, the five lines after the If/Else), in place, fp32:
@@ -173,6 +182,42 @@ int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dty
                        void* stats_out, float* gbar_out, int64_t* b_next_out, float* params,
                        float* m, float* v, const abs_adamw_hparams* hparams, int64_t step,
                        abs_stream_t stream);
+
+/*
+ * The coordinate-wise norm test (Sec. 4: the test Proposition 1 and Theorem 1 are stated for;
+ * Appendix B, first remark, prints it for the exact variance: for every coordinate i,
+ * E[(d_i L_B - d_i L)^2] <= eta^2 (d_i L)^2).  The paper prints no sample form and runs the
+ * summed test in its experiments; this is the sample form obtained the way Eq. 5 is obtained
+ * from the exact-variance test -- coordinate i of the variance estimator displayed before
+ * Eq. 5, divided by b, against eta^2 gbar_i^2:
+ *   T_i = ((1/K) sum_k (g_k[i]-gbar[i])^2) / (eta^2 gbar[i]^2),  T = max_i T_i,
+ *   b_next = ceil(T) if T > b_cur else b_cur
+ * (the smallest batch size under which every coordinate would pass).  A coordinate with zero
+ * variance has T_i = 0, also when gbar[i] = 0; positive variance with gbar[i] = 0 gives +inf.
+ * T is never below the summed statistic of the same data (a weighted mean of the T_i).
+ *
+ * Same arguments as abs_norm_test / abs_normtest_adamw, same gbar, n2, S and (fused) AdamW
+ * update, same traffic: the ratio is formed where the deviations and the mean already are.
+ * What differs in stats_out: the Q slots read NaN; ABS_STAT_T is max_i T_i and
+ * ABS_STAT_ARGMAX the lowest coordinate that attains it; ABS_STAT_FLAGS: NONFINITE (T = NaN,
+ * b kept) when n2 or S is not finite, else DEGENERATE when n2 = 0 or T = +inf, VIOLATED when
+ * T > b_cur; shard record s is {n2_s, S_s, argmax within the shard, max T_i within the shard}.
+ * Accuracy: each ratio is formed in fp32 (hardware reciprocal), so T carries a relative error
+ * of a few 1e-7 for up to 16 workers and up to about 1e-5 beyond (shifted one-pass
+ * deviations); among coordinates whose ratios agree to that accuracy any one may be reported.
+ * Ratios beyond the fp32 range (|gbar[i]| below about 1e-19 times the deviations) are
+ * reported as +inf.
+ */
+int abs_norm_test_coordwise(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                            const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                            void* stats_out, float* gbar_out, int64_t* b_next_out,
+                            abs_stream_t stream);
+int abs_normtest_adamw_coordwise(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                                 const int64_t* shard_offsets, int n_shards, double eta,
+                                 int64_t b_cur, void* stats_out, float* gbar_out,
+                                 int64_t* b_next_out, float* params, float* m, float* v,
+                                 const abs_adamw_hparams* hparams, int64_t step,
+                                 abs_stream_t stream);
 
 /*
  * abs_normtest_adamw for callers that cannot allocate device memory.

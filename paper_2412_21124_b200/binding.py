@@ -21,7 +21,7 @@ ABS_ERR_ALIAS = -8
 ABS_NOALLOC_MAX_CHUNKS = 131072
 ABS_MAX_WORKERS, ABS_MAX_SHARDS = 64, 128
 (ABS_STAT_N2, ABS_STAT_S, ABS_STAT_Q, ABS_STAT_T, ABS_STAT_FLAGS, ABS_STAT_NORM,
- ABS_STAT_NCHUNKS) = range(7)
+ ABS_STAT_NCHUNKS, ABS_STAT_ARGMAX) = range(8)
 ABS_STATS_HEADER, ABS_SHARD_STRIDE = 8, 4
 ABS_FLAG_DEGENERATE, ABS_FLAG_NONFINITE, ABS_FLAG_VIOLATED = 1, 2, 4
 
@@ -48,7 +48,8 @@ def lib():
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB_PATH
+    # ABS_NORMTEST_LIB: a library built elsewhere (another build of the same sources)
+    path = os.environ.get("ABS_NORMTEST_LIB") or _build.LIB_PATH
     if not os.path.exists(path):
         raise RuntimeError(
             "libabs_normtest.so is missing: build it with `python -m paper_2412_21124_b200.build` "
@@ -71,6 +72,12 @@ def lib():
                                      ptr, ptr, ptr, ptr, i64, ptr]
     L.abs_normtest_adamw_noalloc.restype = cint
     L.abs_normtest_adamw_noalloc.argtypes = list(L.abs_normtest_adamw.argtypes)
+    L.abs_norm_test_coordwise.restype = cint
+    L.abs_norm_test_coordwise.argtypes = list(L.abs_norm_test.argtypes)
+    L.abs_norm_test_q.restype = cint
+    L.abs_norm_test_q.argtypes = list(L.abs_norm_test.argtypes)
+    L.abs_normtest_adamw_coordwise.restype = cint
+    L.abs_normtest_adamw_coordwise.argtypes = list(L.abs_normtest_adamw.argtypes)
     L.abs_normtest_adamw_mixed.restype = cint
     L.abs_normtest_adamw_mixed.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64, ptr, ptr,
                                            ptr, ptr, ptr, ptr, ptr, ptr, i64, ptr]
@@ -209,18 +216,32 @@ def alloc_persample_stats(b, d, device="cuda"):
 
 # ------------------------------------------------------------------------- entry points
 def abs_norm_test(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offsets=None,
-                  stream=None):
+                  stream=None, _entry="abs_norm_test"):
     table, K, d, code = _grad_table(grads)
     offs, n_shards = _offsets(shard_offsets)
     _check_f32_vec(gbar_out, d, "gbar_out")
     _check_stats(stats_out, abs_stats_bytes(d, n_shards))
     _check_b_next(b_next_out)
     _check_one_device(*grads, stats_out, gbar_out, b_next_out)
-    rc = lib().abs_norm_test(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
-                             stats_out.data_ptr(), gbar_out.data_ptr(), b_next_out.data_ptr(),
-                             _stream(stream))
+    rc = getattr(lib(), _entry)(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
+                                stats_out.data_ptr(), gbar_out.data_ptr(), b_next_out.data_ptr(),
+                                _stream(stream))
     if rc != ABS_OK:
-        raise AbsError(rc, "abs_norm_test")
+        raise AbsError(rc, _entry)
+
+
+def abs_norm_test_q(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offsets=None,
+                    stream=None):
+    """abs_norm_test that also computes the diagnostic Q = sum_k ||g_k||^2."""
+    abs_norm_test(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offsets, stream,
+                  _entry="abs_norm_test_q")
+
+
+def abs_norm_test_coordwise(grads, eta, b_cur, stats_out, gbar_out, b_next_out,
+                            shard_offsets=None, stream=None):
+    """The coordinate-wise test: T = max_i T_i, its coordinate in the ABS_STAT_ARGMAX slot."""
+    abs_norm_test(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offsets, stream,
+                  _entry="abs_norm_test_coordwise")
 
 
 def abs_adamw_step(params, gbar, m, v, hparams, step, stream=None):
@@ -252,7 +273,7 @@ def abs_adamw_step_clipped(params, gbar, m, v, hparams, step, max_norm, stats_in
 
 
 def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v, hparams,
-                       step, shard_offsets=None, stream=None):
+                       step, shard_offsets=None, stream=None, _entry="abs_normtest_adamw"):
     table, K, d, code = _grad_table(grads)
     offs, n_shards = _offsets(shard_offsets)
     for t, name in ((params, "params"), (m, "m"), (v, "v")):
@@ -263,13 +284,20 @@ def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, param
     _check_b_next(b_next_out)
     _check_one_device(*grads, stats_out, gbar_out, b_next_out, params, m, v)
     hp = _hparams(hparams)
-    rc = lib().abs_normtest_adamw(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
-                                  stats_out.data_ptr(),
-                                  gbar_out.data_ptr() if gbar_out is not None else None,
-                                  b_next_out.data_ptr(), params.data_ptr(), m.data_ptr(),
-                                  v.data_ptr(), ctypes.byref(hp), int(step), _stream(stream))
+    rc = getattr(lib(), _entry)(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
+                                stats_out.data_ptr(),
+                                gbar_out.data_ptr() if gbar_out is not None else None,
+                                b_next_out.data_ptr(), params.data_ptr(), m.data_ptr(),
+                                v.data_ptr(), ctypes.byref(hp), int(step), _stream(stream))
     if rc != ABS_OK:
-        raise AbsError(rc, "abs_normtest_adamw")
+        raise AbsError(rc, _entry)
+
+
+def abs_normtest_adamw_coordwise(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v,
+                                 hparams, step, shard_offsets=None, stream=None):
+    """The fused step with the coordinate-wise test as its decision."""
+    abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v, hparams,
+                       step, shard_offsets, stream, _entry="abs_normtest_adamw_coordwise")
 
 
 def _check_bf16_vec(t, d, name):
@@ -362,7 +390,7 @@ class FusedStep:
     """
 
     def __init__(self, grads, stats_out, gbar_out, b_next_out, params, m, v, hparams,
-                 shard_offsets=None, params_bf16_out=None):
+                 shard_offsets=None, params_bf16_out=None, coordwise=False):
         self._keep = (list(grads), stats_out, gbar_out, b_next_out, params, m, v, params_bf16_out)
         self._table, self._K, self._d, self._code = _grad_table(grads)
         self._offs, self._n_shards = _offsets(shard_offsets)
@@ -377,8 +405,10 @@ class FusedStep:
         self._hp_ref = ctypes.byref(self._hp)
         self._ptrs = (stats_out.data_ptr(), gbar_out.data_ptr() if gbar_out is not None else None,
                       b_next_out.data_ptr(), params.data_ptr(), m.data_ptr(), v.data_ptr())
-        self._fn = lib().abs_normtest_adamw
+        self._fn = lib().abs_normtest_adamw_coordwise if coordwise else lib().abs_normtest_adamw
         self._p16 = None
+        if coordwise and params_bf16_out is not None:
+            raise ValueError("the coordinate-wise step has no mixed-precision variant")
         if params_bf16_out is not None:  # mixed precision: also the bf16 copy of the parameters
             _check_bf16_vec(params_bf16_out, self._d, "params_bf16_out")
             self._p16 = params_bf16_out.data_ptr()
@@ -475,6 +505,9 @@ def read_stats(stats_out, n_shards=1):
     h = stats_out[:n].cpu().tolist()
     shards = [tuple(h[ABS_STATS_HEADER + s * ABS_SHARD_STRIDE + j] for j in range(3))
               for s in range(n_shards)]
+    # fourth slot of a shard record: 0, or the shard's largest T_i (coordinate-wise calls)
+    shard_max = [h[ABS_STATS_HEADER + s * ABS_SHARD_STRIDE + 3] for s in range(n_shards)]
     return {"n2": h[ABS_STAT_N2], "S": h[ABS_STAT_S], "Q": h[ABS_STAT_Q], "T": h[ABS_STAT_T],
             "flags": int(h[ABS_STAT_FLAGS]), "norm": h[ABS_STAT_NORM],
-            "n_chunks": int(h[ABS_STAT_NCHUNKS]), "shards": shards}
+            "n_chunks": int(h[ABS_STAT_NCHUNKS]), "argmax": int(h[ABS_STAT_ARGMAX]),
+            "shards": shards, "shard_max": shard_max}

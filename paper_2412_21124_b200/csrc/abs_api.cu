@@ -9,12 +9,27 @@
 #include <unordered_map>
 #include <utility>
 
-#include "abs_device.cuh"
-#include "normtest_bulk.cuh"
-#include "normtest_stream.cuh"
+#include "launch.cuh"
 #include "persample.cuh"
 
 using namespace absnt;
+
+// The kernels behind these are instantiated in stream_inst.cu, once per combination.
+namespace absnt {
+#define ABS_DECLARE_STREAM(GT, ADAM, STAT) \
+  extern template cudaError_t launch_stream<GT, ADAM, STAT>(const StreamParams&, cudaStream_t);
+ABS_DECLARE_STREAM(F32, true, kStatSums)
+ABS_DECLARE_STREAM(BF16, true, kStatSums)
+ABS_DECLARE_STREAM(F32, false, kStatSumsQ)
+ABS_DECLARE_STREAM(BF16, false, kStatSumsQ)
+ABS_DECLARE_STREAM(F32, false, kStatSums)
+ABS_DECLARE_STREAM(BF16, false, kStatSums)
+ABS_DECLARE_STREAM(F32, true, kStatCoordwise)
+ABS_DECLARE_STREAM(BF16, true, kStatCoordwise)
+ABS_DECLARE_STREAM(F32, false, kStatCoordwise)
+ABS_DECLARE_STREAM(BF16, false, kStatCoordwise)
+#undef ABS_DECLARE_STREAM
+}  // namespace absnt
 
 namespace {
 
@@ -63,25 +78,9 @@ AdamScalars make_adam(const abs_adamw_hparams* h, int64_t step) {
   return a;
 }
 
-// Launch with the programmatic-stream-serialization attribute (see grid_dependency_wait).
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st,
-                       Args&&... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
-}
-
 // Largest cluster (8, 4, 2 or 1 CTAs) of finalize_kernel that the current device can
-// co-schedule, asked once per device and cached.  A refusal (SM partitioning, a shared
+// co-schedule (asked for the variant with the larger shared-memory footprint), asked once per
+// device and cached.  A refusal (SM partitioning, a shared
 // device) or a failing query means 1: a plain single-CTA launch, which cannot be refused for
 // lack of co-scheduling.  The sums do not depend on the cluster size, so the fallback changes
 // no output bit.
@@ -107,7 +106,7 @@ int finalize_max_cluster() {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int active = 0;
-    if (cudaOccupancyMaxActiveClusters(&active, finalize_kernel, &cfg) == cudaSuccess &&
+    if (cudaOccupancyMaxActiveClusters(&active, finalize_kernel<true>, &cfg) == cudaSuccess &&
         active >= 1) {
       best = n;
       break;
@@ -123,7 +122,8 @@ int finalize_max_cluster() {
 // shape of every sum) follows from the chunk counts alone; the cluster size only decides how
 // many warps share the slices.  `max_ctas` is finalize_max_cluster(), queried by the caller
 // before its first launch so that nothing that can be foreseen fails after it.
-cudaError_t launch_finalize(FinalizeParams fp, int max_ctas, cudaStream_t st) {
+cudaError_t launch_finalize(FinalizeParams fp, int max_ctas, cudaStream_t st,
+                            bool coordwise = false) {
   int slice = kFinalizeSlice;
   for (;;) {
     int64_t n = 0;
@@ -156,7 +156,8 @@ cudaError_t launch_finalize(FinalizeParams fp, int max_ctas, cudaStream_t st) {
   attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = n_ctas > 1 ? 2 : 1;  // one CTA: an ordinary launch (its own implicit cluster)
-  return cudaLaunchKernelEx(&cfg, finalize_kernel, fp);
+  return coordwise ? cudaLaunchKernelEx(&cfg, finalize_kernel<true>, fp)
+                   : cudaLaunchKernelEx(&cfg, finalize_kernel<false>, fp);
 }
 
 bool misaligned(const void* p, size_t a) {
@@ -221,150 +222,6 @@ int make_layout(int64_t d, const int64_t* shard_offsets, int n_shards, bool fuse
   return ABS_OK;
 }
 
-// Raises a kernel's dynamic shared-memory limit once per (kernel, device): the attribute call
-// costs about a microsecond of host time, which a launch-bound small-d loop would pay per step.
-cudaError_t allow_dynamic_smem(const void* kernel, size_t smem) {
-  static std::mutex mu;
-  static std::unordered_map<const void*, uint64_t> done;  // kernel -> bit per device
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  const uint64_t bit = dev < 64 ? (uint64_t{1} << dev) : 0;
-  {
-    std::lock_guard<std::mutex> lock(mu);
-    auto it = done.find(kernel);
-    if (bit && it != done.end() && (it->second & bit)) return cudaSuccess;
-  }
-  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(smem));
-  if (e != cudaSuccess) return e;
-  std::lock_guard<std::mutex> lock(mu);
-  done[kernel] |= bit;
-  return cudaSuccess;
-}
-
-// Launch with dynamic shared memory above the 48 KB default.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                            cudaStream_t st, Args&&... args) {
-  cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(kernel), smem);
-  if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
-}
-
-// One (dtype, K) instantiation: the bulk-async kernel where its stages leave room for two or
-// three CTAs per SM, else the register-direct kernel.
-template <typename GT, int KB, bool EXACT, bool ADAM>
-cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
-  const dim3 grid(static_cast<unsigned>(prm.n_chunks));
-  // Measured exceptions.  Fused: the 512-coordinate tile loses to the register-direct kernel
-  // when the worker loop is predicated (EXACT false; K=12: 5.46 vs 5.80 TB/s).  Unfused test
-  // (K*s + 4 bytes per coordinate, so more coordinates per second and more instructions per
-  // byte): staging wins by 1-9% for most worker counts (fp32 K=5 6.39 -> 6.96 TB/s, bf16 K=9
-  // 6.42 -> 6.87) but loses where the register-direct kernel is at its best: one or two
-  // workers (bf16 K=1 -37%, K=2 -7%; fp32 K=2 equal) and bf16 K=6 (-0.4%), K=8 (-2.8%).
-  constexpr BulkShape shape = bulk_shape<GT, KB, ADAM>();
-  constexpr bool kBf16 = std::is_same<GT, BF16>::value;
-  constexpr bool staged_test = EXACT && KB >= 3 && !(kBf16 && (KB == 6 || KB == 8));
-  constexpr int tile = ADAM ? ((shape.tile == 512 && !EXACT) ? 0 : shape.tile)
-                            : (staged_test ? shape.tile : 0);
-  if constexpr (tile > 0) {
-    constexpr size_t smem =
-        static_cast<size_t>(shape.stages) * bulk_stage_bytes<GT, KB, ADAM>(tile);
-    return launch_pdl_smem(
-        normtest_bulk_kernel<GT, KB, EXACT, ADAM, !ADAM, tile, shape.stages, shape.ctas>, grid,
-        dim3(tile / 4), smem, st, prm);
-  } else {
-    return launch_pdl(normtest_stream_kernel<GT, KB, EXACT, ADAM, !ADAM>, grid, dim3(kThreads), st,
-                      prm);
-  }
-}
-
-// More than 16 workers: the split kernel, four coordinates per thread-row (bf16 gradients
-// are then read with 8-byte loads).  KB bounds the worker count of the instantiation.
-template <typename GT, bool EXACT, bool ADAM, int KB = 32>
-cudaError_t launch_split(const StreamParams& prm, cudaStream_t st) {
-  using G4 = typename std::conditional<std::is_same<GT, BF16>::value, BF16H, GT>::type;
-  return launch_pdl(normtest_split_kernel<G4, KB, EXACT, ADAM, !ADAM>,
-                    dim3(static_cast<unsigned>(prm.n_chunks)), dim3(kThreads), st, prm);
-}
-
-// The fused kernel leaves Q out (its stats slot reads NaN): at the power cap the K extra
-// multiply-adds per coordinate cost about 1% of bandwidth.  The unfused test computes it.
-template <typename GT, bool ADAM>
-cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
-  const int K = prm.K;
-  switch (K) {
-    // every count up to 16 has an unrolled kernel of its own (one kernel for a range of counts,
-    // predicating the absent workers, ran 10-25% slower: bf16 K=12 5.6 vs 6.9 TB/s, fp32 K=6
-    // 5.5 vs 7.1)
-    case 1: return launch_one<GT, 1, true, ADAM>(prm, st);
-    case 2: return launch_one<GT, 2, true, ADAM>(prm, st);
-    case 3: return launch_one<GT, 3, true, ADAM>(prm, st);
-    case 4: return launch_one<GT, 4, true, ADAM>(prm, st);
-    case 5: return launch_one<GT, 5, true, ADAM>(prm, st);
-    case 6: return launch_one<GT, 6, true, ADAM>(prm, st);
-    case 7: return launch_one<GT, 7, true, ADAM>(prm, st);
-    case 8: return launch_one<GT, 8, true, ADAM>(prm, st);
-    case 9: return launch_one<GT, 9, true, ADAM>(prm, st);
-    case 10: return launch_one<GT, 10, true, ADAM>(prm, st);
-    case 11: return launch_one<GT, 11, true, ADAM>(prm, st);
-    case 12: return launch_one<GT, 12, true, ADAM>(prm, st);
-    case 13: return launch_one<GT, 13, true, ADAM>(prm, st);
-    case 14: return launch_one<GT, 14, true, ADAM>(prm, st);
-    case 15: return launch_one<GT, 15, true, ADAM>(prm, st);
-    case 16: return launch_one<GT, 16, true, ADAM>(prm, st);
-    case 32: return launch_split<GT, true, ADAM>(prm, st);
-    case 64:  // bf16: four unrolled groups of 16; fp32 spills in that form and takes the loop
-      if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, 64>(prm, st);
-      else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
-    case 17: return launch_split<GT, true, ADAM, 17>(prm, st);
-    case 18: return launch_split<GT, true, ADAM, 18>(prm, st);
-    case 19: return launch_split<GT, true, ADAM, 19>(prm, st);
-    case 20: return launch_split<GT, true, ADAM, 20>(prm, st);
-    case 21: return launch_split<GT, true, ADAM, 21>(prm, st);
-    case 22: return launch_split<GT, true, ADAM, 22>(prm, st);
-    case 23: return launch_split<GT, true, ADAM, 23>(prm, st);
-    case 24: return launch_split<GT, true, ADAM, 24>(prm, st);
-    case 25: return launch_split<GT, true, ADAM, 25>(prm, st);
-    case 26: return launch_split<GT, true, ADAM, 26>(prm, st);
-    case 27: return launch_split<GT, true, ADAM, 27>(prm, st);
-    case 28: return launch_split<GT, true, ADAM, 28>(prm, st);
-    case 29: return launch_split<GT, true, ADAM, 29>(prm, st);
-    case 30: return launch_split<GT, true, ADAM, 30>(prm, st);
-    case 31: return launch_split<GT, true, ADAM, 31>(prm, st);
-    case 48:
-      if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, 48>(prm, st);
-      else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
-#define ABS_SPLIT_BF16_CASE(N)                                                              \
-  case N:                                                                                   \
-    if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, N>(prm, st); \
-    else return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
-    // the multiples of four above 32 (J workers x M accumulation steps is one in practice)
-    ABS_SPLIT_BF16_CASE(36)
-    ABS_SPLIT_BF16_CASE(40)
-    ABS_SPLIT_BF16_CASE(44)
-    ABS_SPLIT_BF16_CASE(52)
-    ABS_SPLIT_BF16_CASE(56)
-    ABS_SPLIT_BF16_CASE(60)
-#undef ABS_SPLIT_BF16_CASE
-    default:
-      // 33..63 workers without a kernel of their own: run-time groups and unpredicated pieces
-      // (5.6-6.1 TB/s; a kernel with compile-time groups runs at 6.4-6.7, as K = 17..32 show)
-      return launch_split<GT, false, ADAM, ABS_MAX_WORKERS>(prm, st);
-  }
-}
-
 // ---------------------------------------------------------------------------------------
 // abs_normtest_adamw_noalloc: the fused step with its chunk records in an array that is
 // part of the library image, for callers that cannot allocate device memory.
@@ -402,7 +259,9 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                   const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
                   void* stats_out, float* gbar_out, int64_t* b_next_out, float* params, float* m,
                   float* v, void* params_bf16, const abs_adamw_hparams* hparams, int64_t step,
-                  bool fused, abs_stream_t stream, bool builtin_records = false) {
+                  bool fused, abs_stream_t stream, bool builtin_records = false,
+                  int stat = -1) {
+  if (stat < 0) stat = kStatSums;
   if (!grads || !stats_out || !b_next_out) return ABS_ERR_NULL;
   if (!fused && !gbar_out) return ABS_ERR_NULL;
   if (fused && (!params || !m || !v)) return ABS_ERR_NULL;
@@ -474,10 +333,22 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
-  if (dtype == ABS_F32)
-    e = fused ? launch_stream<F32, true>(prm, st) : launch_stream<F32, false>(prm, st);
-  else
-    e = fused ? launch_stream<BF16, true>(prm, st) : launch_stream<BF16, false>(prm, st);
+  const bool f32 = dtype == ABS_F32;
+  if (stat == kStatCoordwise) {
+    e = fused ? (f32 ? launch_stream<F32, true, kStatCoordwise>(prm, st)
+                     : launch_stream<BF16, true, kStatCoordwise>(prm, st))
+              : (f32 ? launch_stream<F32, false, kStatCoordwise>(prm, st)
+                     : launch_stream<BF16, false, kStatCoordwise>(prm, st));
+  } else if (fused) {
+    e = f32 ? launch_stream<F32, true, kStatSums>(prm, st)
+            : launch_stream<BF16, true, kStatSums>(prm, st);
+  } else if (stat == kStatSumsQ) {
+    e = f32 ? launch_stream<F32, false, kStatSumsQ>(prm, st)
+            : launch_stream<BF16, false, kStatSumsQ>(prm, st);
+  } else {
+    e = f32 ? launch_stream<F32, false, kStatSums>(prm, st)
+            : launch_stream<BF16, false, kStatSums>(prm, st);
+  }
   if (e != cudaSuccess) return cuda_fail(e);
 
   FinalizeParams fp;
@@ -491,7 +362,8 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   fp.eta = eta;
   fp.norm = static_cast<double>(K);
   fp.b_cur = b_cur;
-  e = launch_finalize(fp, finalize_ctas, st);
+  std::memcpy(fp.shard_first, L.shard_off, sizeof(int64_t) * L.n_shards);
+  e = launch_finalize(fp, finalize_ctas, st, stat == kStatCoordwise);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }
@@ -551,6 +423,14 @@ int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                        stream);
 }
 
+int abs_norm_test_q(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                    const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                    void* stats_out, float* gbar_out, int64_t* b_next_out, abs_stream_t stream) {
+  return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
+                       gbar_out, b_next_out, nullptr, nullptr, nullptr, nullptr, nullptr, 0, false,
+                       stream, false, kStatSumsQ);
+}
+
 int abs_normtest_adamw(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                        const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
                        void* stats_out, float* gbar_out, int64_t* b_next_out, float* params,
@@ -569,6 +449,26 @@ int abs_normtest_adamw_mixed(const void* const* grads, int K, int64_t d, abs_dty
   return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
                        gbar_out, b_next_out, params, m, v, params_bf16_out, hparams, step, true,
                        stream);
+}
+
+int abs_norm_test_coordwise(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                            const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
+                            void* stats_out, float* gbar_out, int64_t* b_next_out,
+                            abs_stream_t stream) {
+  return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
+                       gbar_out, b_next_out, nullptr, nullptr, nullptr, nullptr, nullptr, 0, false,
+                       stream, false, kStatCoordwise);
+}
+
+int abs_normtest_adamw_coordwise(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                                 const int64_t* shard_offsets, int n_shards, double eta,
+                                 int64_t b_cur, void* stats_out, float* gbar_out,
+                                 int64_t* b_next_out, float* params, float* m, float* v,
+                                 const abs_adamw_hparams* hparams, int64_t step,
+                                 abs_stream_t stream) {
+  return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
+                       gbar_out, b_next_out, params, m, v, nullptr, hparams, step, true, stream,
+                       false, kStatCoordwise);
 }
 
 namespace {

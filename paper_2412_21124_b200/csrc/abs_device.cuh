@@ -46,6 +46,7 @@ struct FinalizeParams {
   const double* chunk_in;
   int32_t chunk_prefix[ABS_MAX_SHARDS + 1];
   int32_t slice_prefix[ABS_MAX_SHARDS + 1];  // slices of `slice` records before each shard
+  int64_t shard_first[ABS_MAX_SHARDS];       // first coordinate of each shard (coordinate-wise test)
   int slice;                                 // records per slice
   int n_shards;
   int n_chunks;

@@ -137,9 +137,11 @@ struct BulkGrad<F32> {
   }
 };
 
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ, int TILE, int STAGES, int CTAS>
+template <typename GT, int KB, bool EXACT, bool ADAM, int STAT, int TILE, int STAGES, int CTAS>
 __global__ void __launch_bounds__(TILE / 4, CTAS)
     normtest_bulk_kernel(const __grid_constant__ StreamParams prm) {
+  constexpr bool WITHQ = STAT == kStatSumsQ;
+  constexpr bool CW = STAT == kStatCoordwise;
   constexpr int kBulkTile = TILE;
   constexpr int kBulkStages = STAGES;
   constexpr int NT = TILE / 4;  // threads
@@ -173,10 +175,13 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
       waited = true;
     }
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
+    CwMax cw;
+    cw.init(tid * 4);
     const bool bulk = cg.aligned && (cg.hi - cg.lo == prm.chunk_elems) &&
                       (prm.chunk_elems % kBulkTile == 0);
     if (!bulk) {
-      chunk_rows_direct<GT, KB, EXACT, ADAM, WITHQ, NT>(prm, K, cg, acc_n2, acc_S, acc_Q);
+      cw.init(tid * GT::kVec);
+      chunk_rows_direct<GT, KB, EXACT, ADAM, STAT, NT>(prm, K, cg, acc_n2, acc_S, acc_Q, cw);
     } else {
       const int n_tiles = prm.chunk_elems / kBulkTile;
       const uint32_t tx_bytes = static_cast<uint32_t>(K * GB + (ADAM ? 3 * FB : 0));
@@ -244,6 +249,11 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
           row_S += dev2.y;
           row_Q += sq.x;
           row_Q += sq.y;
+          if (CW) {
+            const int li = i * kBulkTile + tid * 4 + 2 * jp;
+            cw.update(dev2.x, mean.x, li);
+            cw.update(dev2.y, mean.y, li + 1);
+          }
           if (ADAM) adamw_pair(prm.adam, mean, w2[jp], m2[jp], v2[jp]);
         }
         acc_n2 += static_cast<double>(row_n2);
@@ -281,7 +291,7 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
       if (tid == 0) bulk_wait_stores_read();
     }
     if (lost) acc_S = __longlong_as_double(0x7ff8000000000000ll);  // poison: a copy was lost
-    write_chunk_record<WITHQ, NT>(prm, chunk, acc_n2, acc_S, acc_Q, red);
+    write_chunk_record<STAT, NT>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, cw, red);
   }
   if (tid == 0) {
     bulk_wait_stores_done();

@@ -29,6 +29,42 @@
 
 namespace absnt {
 
+// What a kernel accumulates besides gbar: the two sums of the test always; the diagnostic
+// Q = sum_k ||g_k||^2 on request; or, for the coordinate-wise test (Sec. 4, Proposition 1),
+// the largest per-coordinate ratio sum_k (g_k[i]-gbar_i)^2 / gbar_i^2 and where it occurs.
+enum StatMode { kStatSums = 0, kStatSumsQ = 1, kStatCoordwise = 2 };
+
+// Running maximum of the per-coordinate ratio within one thread, then one chunk.  The ratio is
+// formed in fp32 with the hardware reciprocal (2^-22 relative).  A coordinate with zero
+// deviations and zero mean gives 0 * inf = NaN, one with a non-finite input gives NaN as well:
+// NaN never compares greater, so such coordinates are skipped here (non-finite inputs are
+// reported through the sums).  Zero mean with positive deviations gives +inf.  Ties keep the
+// lower index: a thread visits its coordinates in increasing order and replaces only on a
+// strictly greater ratio.
+struct CwMax {
+  float r;
+  int idx;  // coordinate index relative to the chunk's first coordinate
+  __device__ __forceinline__ void init(int first_idx) {
+    r = 0.f;
+    idx = first_idx;
+  }
+  __device__ __forceinline__ void update(float dev2, float mean, int i) {
+    float inv;
+    asm("rcp.approx.f32 %0, %1;" : "=f"(inv) : "f"(mean * mean));
+    const float q = dev2 * inv;
+    if (q > r) {
+      r = q;
+      idx = i;
+    }
+  }
+  __device__ __forceinline__ void merge(float r2, int idx2) {
+    if (r2 > r || (r2 == r && idx2 < idx)) {
+      r = r2;
+      idx = idx2;
+    }
+  }
+};
+
 // Mean, squared deviations and (optionally) squared values of one coordinate.
 template <typename GT, int KB, bool EXACT, bool WITHQ>
 __device__ __forceinline__ float coord_math(const float (&g)[KB], int K, const StreamParams& prm,
@@ -136,10 +172,13 @@ __device__ __forceinline__ float coord_math_split(const float (&g)[KB], int K,
 // rows that are ragged (end of a shard) or whose streams are not 16-byte aligned.  Same
 // arithmetic in the same order as the vector path, so both give identical bits.  Kept out
 // of line so that its registers do not weigh on the vector path.
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ, bool SPLIT = false>
+template <typename GT, int KB, bool EXACT, bool ADAM, int STAT, bool SPLIT = false>
 __device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t base, int64_t hi,
-                                        float* sums /* n2, S, Q of this thread-row */) {
+                                        int64_t chunk_lo,
+                                        float* sums /* n2, S, Q of this thread-row */,
+                                        CwMax* cw) {
   constexpr int V = GT::kVec;
+  constexpr bool WITHQ = STAT == kStatSumsQ;
   float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
   for (int e = 0; e < V; ++e) {
     const int64_t i = base + e;
@@ -153,6 +192,7 @@ __device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t 
     row_n2 = fmaf(mean, mean, row_n2);
     row_S += dev2;
     row_Q += sq;
+    if (STAT == kStatCoordwise) cw->update(dev2, mean, static_cast<int>(i - chunk_lo));
     if (prm.gbar) prm.gbar[i] = mean;
     if (ADAM) {
       float w = prm.p[i], m = prm.m[i], v = prm.v[i];
@@ -209,11 +249,13 @@ __device__ __forceinline__ ChunkGeometry chunk_geometry(const StreamParams& prm,
 
 // Register-direct processing of one chunk: every thread-row is loaded with 128/256-bit
 // global loads straight into registers.  Adds this thread's sums to acc_*.
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ, int NT = kThreads>
+template <typename GT, int KB, bool EXACT, bool ADAM, int STAT, int NT = kThreads>
 __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K,
                                                   const ChunkGeometry& cg, double& acc_n2,
-                                                  double& acc_S, double& acc_Q) {
+                                                  double& acc_S, double& acc_Q, CwMax& cw) {
   constexpr int V = GT::kVec;
+  constexpr bool WITHQ = STAT == kStatSumsQ;
+  constexpr bool CW = STAT == kStatCoordwise;
   constexpr int NF4 = V / 4; // float4 per thread-row of an fp32 array
   // 256-bit stores of the fp32 arrays pay off for few workers (K <= 7: +3..9% measured) and
   // cost about 1% for K >= 8, where the stores of the first half are better issued early;
@@ -261,6 +303,7 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
             row_n2 = fmaf(mean, mean, row_n2);
             row_S += dev2;
             row_Q += sq;
+            if (CW) cw.update(dev2, mean, static_cast<int>(base - cg.lo) + 4 * q + j);
           }
           gbv[q] = make_float4(gb[0], gb[1], gb[2], gb[3]);
         }
@@ -312,9 +355,13 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
 #pragma unroll
       for (int q = 0; q < NF4; ++q) {
         float gb[4];
-        if constexpr (ADAM) {
-          // fused: two coordinates per packed fp32 instruction (+0.4..0.8% at K = 16); the row
-          // sums take the coordinates in index order, as scalar_row does
+        // Two coordinates per packed fp32 instruction in the fused kernels (+0.4..0.8% at
+        // K = 16) and in the plain bf16 test with six workers (6.53 -> 6.62 TB/s; with eight it
+        // costs 0.5%, and with Q computed the eight-vector kernels spill: bf16 K=2 6.5 -> 5.8
+        // TB/s).  The row sums take the coordinates in index order, as scalar_row does.
+        constexpr bool kPackedRow =
+            ADAM || (STAT == kStatSums && EXACT && KB == 6 && GT::kVec == 8);
+        if constexpr (kPackedRow) {
           float2* w2 = reinterpret_cast<float2*>(&pw[q]);
           float2* m2 = reinterpret_cast<float2*>(&pm[q]);
           float2* v2 = reinterpret_cast<float2*>(&pv[q]);
@@ -334,11 +381,14 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
             row_S += dev2.y;
             row_Q += sq.x;
             row_Q += sq.y;
-            adamw_pair(prm.adam, mean, w2[jp], m2[jp], v2[jp]);
+            if (CW) {
+              const int li = static_cast<int>(base - cg.lo) + 4 * q + 2 * jp;
+              cw.update(dev2.x, mean.x, li);
+              cw.update(dev2.y, mean.y, li + 1);
+            }
+            if constexpr (ADAM) adamw_pair(prm.adam, mean, w2[jp], m2[jp], v2[jp]);
           }
         } else {
-          // the test alone keeps the scalar form: with the packed one the compiler spills in
-          // the eight-vector kernels (bf16 K=2: 6.5 -> 5.8 TB/s, K=16: -1%)
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             float g[KB];
@@ -351,6 +401,7 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
             row_n2 = fmaf(mean, mean, row_n2);
             row_S += dev2;
             row_Q += sq;
+            if (CW) cw.update(dev2, mean, static_cast<int>(base - cg.lo) + 4 * q + j);
           }
         }
         if (kWideStores && wide) {
@@ -380,7 +431,7 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
       }
     } else if (base < hi) {
       float sums[3];
-      scalar_row<GT, KB, EXACT, ADAM, WITHQ>(prm, K, base, hi, sums);
+      scalar_row<GT, KB, EXACT, ADAM, STAT>(prm, K, base, hi, cg.lo, sums, &cw);
       row_n2 = sums[0];
       row_S = sums[1];
       row_Q = sums[2];
@@ -391,21 +442,48 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
   }
 }
 
-// CTA-wide fixed-order reduction of the per-thread sums and the chunk record.
-template <bool WITHQ, int NT = kThreads>
-__device__ __forceinline__ void write_chunk_record(const StreamParams& prm, int chunk, double acc_n2,
-                                                   double acc_S, double acc_Q, double* red) {
-  block_reduce3<NT / 32>(acc_n2, acc_S, acc_Q, red);
+// CTA-wide fixed-order reduction of the per-thread sums and the chunk record {n2, S, Q, 0}.
+// Coordinate-wise mode: {n2, S, index of the chunk's largest ratio, that ratio}; the maximum
+// is exact and order-independent, ties go to the lower index.
+template <int STAT, int NT = kThreads>
+__device__ __forceinline__ void write_chunk_record(const StreamParams& prm, int chunk,
+                                                   int64_t chunk_lo, double acc_n2, double acc_S,
+                                                   double acc_Q, CwMax cw, double* red) {
+  constexpr bool WITHQ = STAT == kStatSumsQ;
+  constexpr bool CW = STAT == kStatCoordwise;
+  __shared__ float cw_r[NT / 32];
+  __shared__ int cw_i[NT / 32];
+  if (CW) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float r2 = __shfl_down_sync(0xffffffffu, cw.r, off);
+      const int i2 = __shfl_down_sync(0xffffffffu, cw.idx, off);
+      cw.merge(r2, i2);
+    }
+    if ((threadIdx.x & 31) == 0) {
+      cw_r[threadIdx.x >> 5] = cw.r;
+      cw_i[threadIdx.x >> 5] = cw.idx;
+    }
+  }
+  block_reduce3<NT / 32>(acc_n2, acc_S, acc_Q, red);  // synchronises the CTA twice
   if (threadIdx.x == 0) {
     double* out = prm.chunk_out + static_cast<int64_t>(chunk) * 4;
     out[0] = acc_n2;
     out[1] = acc_S;
-    out[2] = WITHQ ? acc_Q : __longlong_as_double(0x7ff8000000000000ll);  // NaN: not computed
-    out[3] = 0.0;
+    if (CW) {
+#pragma unroll
+      for (int w = 1; w < NT / 32; ++w) cw.merge(cw_r[w], cw_i[w]);
+      out[2] = static_cast<double>(chunk_lo + cw.idx);
+      out[3] = static_cast<double>(cw.r);
+    } else {
+      out[2] = WITHQ ? acc_Q : __longlong_as_double(0x7ff8000000000000ll);  // NaN: not computed
+      out[3] = 0.0;
+    }
   }
+  if (CW) __syncthreads();  // cw_r / cw_i are free again before a next chunk's warps write them
 }
 
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+template <typename GT, int KB, bool EXACT, bool ADAM, int STAT>
 __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : ((KB <= 16 || GT::kVec * sizeof(typename GT::scalar) <= 8) ? 2 : 1)))
     normtest_stream_kernel(const __grid_constant__ StreamParams prm) {
   __shared__ double red[kWarps * 3];
@@ -418,8 +496,10 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : ((KB <= 16
       waited = true;
     }
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
-    chunk_rows_direct<GT, KB, EXACT, ADAM, WITHQ>(prm, K, cg, acc_n2, acc_S, acc_Q);
-    write_chunk_record<WITHQ>(prm, chunk, acc_n2, acc_S, acc_Q, red);
+    CwMax cw;
+    cw.init(static_cast<int>(threadIdx.x) * GT::kVec);
+    chunk_rows_direct<GT, KB, EXACT, ADAM, STAT>(prm, K, cg, acc_n2, acc_S, acc_Q, cw);
+    write_chunk_record<STAT>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, cw, red);
   }
 }
 
@@ -429,11 +509,13 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : ((KB <= 16
 // coord_math_split, so only one group of gradient vectors is live per thread (two or three
 // CTAs per SM instead of one at 255 registers, and no instructions for absent workers
 // beyond the last group).
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+template <typename GT, int KB, bool EXACT, bool ADAM, int STAT>
 __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
                                                  const ChunkGeometry& cg, double& acc_n2,
-                                                 double& acc_S, double& acc_Q) {
+                                                 double& acc_S, double& acc_Q, CwMax& cw) {
   constexpr int V = GT::kVec;
+  constexpr bool WITHQ = STAT == kStatSumsQ;
+  constexpr bool CW = STAT == kStatCoordwise;
   static_assert(V == 4, "split path: four coordinates per thread-row");
   // exact K: compile-time groups of 16 and one group of K mod 16; any other K: a run-time loop
   // over groups of 32 bytes
@@ -541,10 +623,16 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
         gb[2 * pi + 1] = mean.y;
         row_n2 = fmaf(mean.x, mean.x, row_n2);
         row_n2 = fmaf(mean.y, mean.y, row_n2);
-        row_S += clamp_nonneg(t.x);
-        row_S += clamp_nonneg(t.y);
+        const float tx = clamp_nonneg(t.x), ty = clamp_nonneg(t.y);
+        row_S += tx;
+        row_S += ty;
         row_Q += q[pi].x;
         row_Q += q[pi].y;
+        if (CW) {
+          const int li = static_cast<int>(base - cg.lo) + 2 * pi;
+          cw.update(tx, mean.x, li);
+          cw.update(ty, mean.y, li + 1);
+        }
         if (ADAM) adamw_pair(prm.adam, mean, w2[pi], m2[pi], v2[pi]);
       }
       if (prm.gbar) st_stream_16(prm.gbar + base, make_float4(gb[0], gb[1], gb[2], gb[3]));
@@ -556,7 +644,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
       }
     } else if (base < hi) {
       float sums[3];
-      scalar_row<GT, KB, EXACT, ADAM, WITHQ, true>(prm, K, base, hi, sums);
+      scalar_row<GT, KB, EXACT, ADAM, STAT, true>(prm, K, base, hi, cg.lo, sums, &cw);
       row_n2 = sums[0];
       row_S = sums[1];
       row_Q = sums[2];
@@ -567,7 +655,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
   }
 }
 
-template <typename GT, int KB, bool EXACT, bool ADAM, bool WITHQ>
+template <typename GT, int KB, bool EXACT, bool ADAM, int STAT>
 __global__ void __launch_bounds__(kThreads, 2)
     normtest_split_kernel(const __grid_constant__ StreamParams prm) {
   __shared__ double red[kWarps * 3];
@@ -580,8 +668,10 @@ __global__ void __launch_bounds__(kThreads, 2)
       waited = true;
     }
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
-    chunk_rows_split<GT, KB, EXACT, ADAM, WITHQ>(prm, K, cg, acc_n2, acc_S, acc_Q);
-    write_chunk_record<WITHQ>(prm, chunk, acc_n2, acc_S, acc_Q, red);
+    CwMax cw;
+    cw.init(static_cast<int>(threadIdx.x) * GT::kVec);
+    chunk_rows_split<GT, KB, EXACT, ADAM, STAT>(prm, K, cg, acc_n2, acc_S, acc_Q, cw);
+    write_chunk_record<STAT>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, cw, red);
   }
 }
 
@@ -608,43 +698,91 @@ constexpr int kFinalizeSlicesPerCta = 16;  // another CTA (another SM's L2 port)
 // records c0 + first, c0 + first + stride, ... (< c1), added in that order.  Each pass issues
 // four unconditional loads (an index past the end re-reads the pass's first record and its
 // values are replaced by +0.0, which leaves the sums unchanged) before the first add.
+// CW: the third and fourth slot of a record are {index, ratio} of the chunk's largest
+// per-coordinate ratio; (c, m) then carry the running {index, ratio} maximum instead of a sum.
+template <bool CW>
 __device__ __forceinline__ void strided_records(const double* chunk_in, int c0, int c1, int first,
-                                                int stride, double& a, double& b, double& c) {
+                                                int stride, double& a, double& b, double& c,
+                                                double& m) {
   constexpr int kInFlight = 4;
   for (int ch = c0 + first; ch < c1; ch += kInFlight * stride) {
-    double2 t[kInFlight];
-    double u2[kInFlight];
+    double2 t[kInFlight], u2[kInFlight];
 #pragma unroll
     for (int u = 0; u < kInFlight; ++u) {
       const int r = ch + u * stride;
       const double* rec = chunk_in + static_cast<int64_t>(r < c1 ? r : ch) * 4;
       t[u] = __ldcg(reinterpret_cast<const double2*>(rec));
-      u2[u] = __ldcg(rec + 2);
+      u2[u] = __ldcg(reinterpret_cast<const double2*>(rec + 2));
     }
 #pragma unroll
     for (int u = 0; u < kInFlight; ++u) {
       const bool live = ch + u * stride < c1;
       a += live ? t[u].x : 0.0;
       b += live ? t[u].y : 0.0;
-      c += live ? u2[u] : 0.0;
+      if (CW) {
+        if (live && (u2[u].y > m || (u2[u].y == m && u2[u].x < c))) {
+          m = u2[u].y;
+          c = u2[u].x;
+        }
+      } else {
+        c += live ? u2[u].x : 0.0;
+      }
     }
   }
 }
 
-__device__ __forceinline__ void warp_tree3(double& a, double& b, double& c) {
+template <bool CW>
+__device__ __forceinline__ void warp_tree3(double& a, double& b, double& c, double& m) {
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
     a += __shfl_down_sync(0xffffffffu, a, off);
     b += __shfl_down_sync(0xffffffffu, b, off);
-    c += __shfl_down_sync(0xffffffffu, c, off);
+    const double c2 = __shfl_down_sync(0xffffffffu, c, off);
+    if (CW) {
+      const double m2 = __shfl_down_sync(0xffffffffu, m, off);
+      if (m2 > m || (m2 == m && c2 < c)) {
+        m = m2;
+        c = c2;
+      }
+    } else {
+      c += c2;
+    }
   }
 }
 
+// The decision of the coordinate-wise test from the largest per-coordinate ratio
+// rmax = max_i sum_k (g_k[i]-gbar_i)^2 / gbar_i^2:  T = (rmax/norm) / eta^2.
+__device__ __forceinline__ int64_t decide_coordwise_device(double S, double n2, double rmax,
+                                                           double norm, double eta, int64_t b_cur,
+                                                           double* T_out, int* flags_out) {
+  int flags = 0;
+  double T = (rmax / norm) / (eta * eta);
+  int64_t b_next = b_cur;
+  if (!isfinite(S) || !isfinite(n2)) {
+    flags |= ABS_FLAG_NONFINITE;
+    T = __longlong_as_double(0x7ff8000000000000ll);
+  } else {
+    if (n2 == 0.0 || isinf(T)) flags |= ABS_FLAG_DEGENERATE;
+    if (T > static_cast<double>(b_cur)) {
+      flags |= ABS_FLAG_VIOLATED;
+      b_next = (T >= 4611686018427387904.0) ? INT64_MAX : static_cast<int64_t>(ceil(T));
+    }
+  }
+  *T_out = T;
+  *flags_out = flags;
+  return b_next;
+}
+
+// CW: the coordinate-wise test (chunk records carry {n2, S, index, ratio}); the shard records
+// written are {n2_s, S_s, index of the shard's largest T_i, that T_i}, the header's Q slot
+// reads NaN, its T slot the largest T_i and its ABS_STAT_ARGMAX slot where it occurs.
+template <bool CW>
 __global__ void __launch_bounds__(kFinalizeThreads)
     finalize_kernel(const __grid_constant__ FinalizeParams fp) {
   namespace cg = cooperative_groups;
-  __shared__ double part[kFinalizeMaxSlices * 3];  // used in CTA 0 only
-  __shared__ double shard_tot[ABS_MAX_SHARDS * 3];
+  constexpr int PS = CW ? 4 : 3;                    // doubles per partial
+  __shared__ double part[kFinalizeMaxSlices * PS];  // used in CTA 0 only
+  __shared__ double shard_tot[ABS_MAX_SHARDS * PS];
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = static_cast<int>(cluster.block_rank());
   const int n_warps = static_cast<int>(cluster.num_blocks()) * kFinalizeWarps;
@@ -666,48 +804,86 @@ __global__ void __launch_bounds__(kFinalizeThreads)
     }
     const int c0 = fp.chunk_prefix[lo] + (i - fp.slice_prefix[lo]) * fp.slice;
     const int c1 = min(c0 + fp.slice, fp.chunk_prefix[lo + 1]);
-    double a = 0.0, b = 0.0, c = 0.0;
-    strided_records(fp.chunk_in, c0, c1, lane, 32, a, b, c);
-    warp_tree3(a, b, c);
+    double a = 0.0, b = 0.0, c = 0.0, m = -1.0;
+    strided_records<CW>(fp.chunk_in, c0, c1, lane, 32, a, b, c, m);
+    warp_tree3<CW>(a, b, c, m);
     if (lane == 0) {
-      part0[3 * i + 0] = a;
-      part0[3 * i + 1] = b;
-      part0[3 * i + 2] = c;
+      part0[PS * i + 0] = a;
+      part0[PS * i + 1] = b;
+      part0[PS * i + 2] = c;
+      if (CW) part0[PS * i + 3] = m;
     }
   }
   // arrive.release / wait.acquire at cluster scope: every partial is visible to CTA 0
   cluster.sync();
   if (rank != 0) return;
   for (int s = warp; s < fp.n_shards; s += kFinalizeWarps) {
-    double a = 0.0, b = 0.0, c = 0.0;
+    double a = 0.0, b = 0.0, c = 0.0, m = -1.0;
     for (int i = fp.slice_prefix[s] + lane; i < fp.slice_prefix[s + 1]; i += 32) {
-      a += part[3 * i + 0];
-      b += part[3 * i + 1];
-      c += part[3 * i + 2];
+      a += part[PS * i + 0];
+      b += part[PS * i + 1];
+      if (CW) {
+        const double m2 = part[PS * i + 3], c2 = part[PS * i + 2];
+        if (m2 > m || (m2 == m && c2 < c)) {
+          m = m2;
+          c = c2;
+        }
+      } else {
+        c += part[PS * i + 2];
+      }
     }
-    warp_tree3(a, b, c);
+    warp_tree3<CW>(a, b, c, m);
     if (lane == 0) {
       double* rec = fp.stats + ABS_STATS_HEADER + s * ABS_SHARD_STRIDE;
       rec[0] = a;
       rec[1] = b;
-      rec[2] = c;
-      rec[3] = 0.0;
-      shard_tot[3 * s + 0] = a;
-      shard_tot[3 * s + 1] = b;
-      shard_tot[3 * s + 2] = c;
+      if (CW) {
+        // an empty shard has no coordinate: ratio 0 at its (empty) start
+        if (m < 0.0) {
+          m = 0.0;
+          c = static_cast<double>(fp.shard_first[s]);
+        }
+        rec[2] = c;
+        rec[3] = (m / fp.norm) / (fp.eta * fp.eta);
+      } else {
+        rec[2] = c;
+        rec[3] = 0.0;
+      }
+      shard_tot[PS * s + 0] = a;
+      shard_tot[PS * s + 1] = b;
+      shard_tot[PS * s + 2] = c;
+      if (CW) shard_tot[PS * s + 3] = m;
     }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    double tot_n2 = 0.0, tot_S = 0.0, tot_Q = 0.0;
+    double tot_n2 = 0.0, tot_S = 0.0, tot_Q = 0.0, rmax = 0.0, arg = 0.0;
+    bool any = false;
     for (int s = 0; s < fp.n_shards; ++s) {
-      tot_n2 += shard_tot[3 * s + 0];
-      tot_S += shard_tot[3 * s + 1];
-      tot_Q += shard_tot[3 * s + 2];
+      tot_n2 += shard_tot[PS * s + 0];
+      tot_S += shard_tot[PS * s + 1];
+      if (CW) {
+        // shards in index order: a later shard wins only with a strictly larger ratio, so a
+        // tie keeps the lower coordinate; empty shards do not take part
+        const bool nonempty = fp.chunk_prefix[s + 1] > fp.chunk_prefix[s];
+        if (nonempty && (!any || shard_tot[PS * s + 3] > rmax)) {
+          rmax = shard_tot[PS * s + 3];
+          arg = shard_tot[PS * s + 2];
+          any = true;
+        }
+      } else {
+        tot_Q += shard_tot[PS * s + 2];
+      }
     }
     double T;
     int flags;
-    const int64_t b_next = decide_device(tot_S, tot_n2, fp.norm, fp.eta, fp.b_cur, &T, &flags);
+    int64_t b_next;
+    if (CW) {
+      b_next = decide_coordwise_device(tot_S, tot_n2, rmax, fp.norm, fp.eta, fp.b_cur, &T, &flags);
+      tot_Q = __longlong_as_double(0x7ff8000000000000ll);
+    } else {
+      b_next = decide_device(tot_S, tot_n2, fp.norm, fp.eta, fp.b_cur, &T, &flags);
+    }
     fp.stats[ABS_STAT_N2] = tot_n2;
     fp.stats[ABS_STAT_S] = tot_S;
     fp.stats[ABS_STAT_Q] = tot_Q;
@@ -715,7 +891,7 @@ __global__ void __launch_bounds__(kFinalizeThreads)
     fp.stats[ABS_STAT_FLAGS] = static_cast<double>(flags);
     fp.stats[ABS_STAT_NORM] = fp.norm;
     fp.stats[ABS_STAT_NCHUNKS] = static_cast<double>(fp.n_chunks);
-    fp.stats[7] = 0.0;
+    fp.stats[ABS_STAT_ARGMAX] = CW ? arg : 0.0;
     *fp.b_next = b_next;
   }
 }

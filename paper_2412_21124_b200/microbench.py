@@ -52,7 +52,7 @@ def bytes_per_call(call, d, K, esz, gbar, b):
 
 
 def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b=4096, dev="cuda",
-              graph=None, mixed=False):
+              graph=None, mixed=False, coordwise=False, with_q=False):
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     esz = 2 if dtype == "bf16" else 4
     nbytes = bytes_per_call(call, d, K, esz, gbar, b)
@@ -86,7 +86,7 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
         if call == "fused":  # marshal once; each timed call is then a single C call
             s["prepared"] = B.FusedStep(s["grads"], s["stats"], s.get("gbar"), s["b_next"], s["p"],
                                         s["m"], s["v"], HP, shard_offsets=offs,
-                                        params_bf16_out=s.get("p16"))
+                                        params_bf16_out=s.get("p16"), coordwise=coordwise)
         sets.append(s)
 
     def one(i):
@@ -94,8 +94,9 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
         if call == "fused":
             s["prepared"].run(0.1, 512, 100 + i)
         elif call == "normtest":
-            B.abs_norm_test(s["grads"], 0.1, 512, s["stats"], s["gbar"], s["b_next"],
-                            shard_offsets=offs)
+            fn = (B.abs_norm_test_coordwise if coordwise
+                  else (B.abs_norm_test_q if with_q else B.abs_norm_test))
+            fn(s["grads"], 0.1, 512, s["stats"], s["gbar"], s["b_next"], shard_offsets=offs)
         elif call == "adamw" and mixed:
             B.abs_adamw_step_mixed(s["p"], s["gbar"], s["m"], s["v"], s["p16"], HP, 100 + i)
         elif call == "adamw":
@@ -157,7 +158,8 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
     sampler.stop()
     ms = e0.elapsed_time(e1) / steps
     out = {"call": call, "d": d, "K": K, "dtype": dtype, "n_shards": n_shards, "gbar": bool(gbar),
-           "mixed": bool(mixed), "steps": steps, "buffer_sets": n_sets, "cuda_graph": bool(graph),
+           "mixed": bool(mixed), "coordwise": bool(coordwise), "with_q": bool(with_q),
+           "steps": steps, "buffer_sets": n_sets, "cuda_graph": bool(graph),
            "ms": ms,
            "bytes": nbytes, "GBps": nbytes / (ms * 1e-3) / 1e9}
     if call == "persample":
@@ -184,6 +186,12 @@ REPORT_POINTS = (
     + [("fused", GPT2, K, "bf16", 1, {}) for K in (6, 12, 20, 24, 27, 31, 36, 40, 44, 48, 52, 56,
                                                    60, 64)]
     + [("fused", GPT2, K, "f32", 1, {}) for K in (12, 20, 31, 48, 64)]
+    # the diagnostic variant and the coordinate-wise test
+    + [("normtest", GPT2, 8, "bf16", 1, {"q": True}), ("normtest", GPT2, 32, "bf16", 1, {"q": True}),
+       ("normtest", GPT2, 8, "bf16", 1, {"coordwise": True}),
+       ("fused", GPT2, 8, "bf16", 1, {"coordwise": True}),
+       ("fused", GPT2, 4, "f32", 1, {"coordwise": True}),
+       ("fused", GPT2, 32, "bf16", 1, {"coordwise": True})]
     # the paper's own model sizes (Table 4), J = 4 workers, bf16
     + [("fused", d, 4, "bf16", 1, {}) for d in (304_600_000, 1_100_000_000, 3_400_000_000)])
 
@@ -207,7 +215,8 @@ def report(args, graph):
     sweep(args, graph)
     for call, d, K, dtype, shards, extra in REPORT_POINTS:
         r = run_point(call, d, K, dtype, shards, args.steps, args.warmup, extra.get("gbar", False),
-                      extra.get("b", 4096), graph=graph, mixed=extra.get("mixed", False))
+                      extra.get("b", 4096), graph=graph, mixed=extra.get("mixed", False),
+                      coordwise=extra.get("coordwise", False), with_q=extra.get("q", False))
         print(json.dumps(r), flush=True)
         torch.cuda.empty_cache()
 
@@ -254,7 +263,8 @@ def format_markdown(path):
         if r.get("sweep"):
             continue
         name = r["call"] + (" +gbar" if r.get("gbar") and r["call"] == "fused" else "") + (
-            " +bf16 copy" if r.get("mixed") else "")
+            " +bf16 copy" if r.get("mixed") else "") + (" +Q" if r.get("with_q") else "") + (
+            " coordinate-wise" if r.get("coordwise") else "")
         kb = r["b"] if r["call"] == "persample" else (r["K"] if r["call"] != "adamw" else "-")
         mhz, why = clk(r)
         print("| %s | %d | %s | %s | %d | %.4f | %.0f | %.3f | %s | %s | %s |" % (
@@ -275,6 +285,10 @@ def main(argv=None):
     ap.add_argument("--gbar", action="store_true", help="fused: also write gbar")
     ap.add_argument("--mixed", action="store_true",
                     help="fused / adamw: also write the bf16 copy of the parameters")
+    ap.add_argument("--q", action="store_true",
+                    help="normtest: abs_norm_test_q (also the diagnostic Q)")
+    ap.add_argument("--coordwise", action="store_true",
+                    help="fused / normtest: the coordinate-wise test as the decision")
     ap.add_argument("--sweep", action="store_true", help="fused call over the d x K x dtype grid")
     ap.add_argument("--report", action="store_true",
                     help="the grid and the per-call points quoted beside it, in one run")
@@ -297,7 +311,8 @@ def main(argv=None):
     else:
         print(json.dumps(run_point(args.call, args.d, args.K, args.dtype, args.shards, args.steps,
                                    args.warmup, args.gbar, args.b, graph=graph,
-                                   mixed=args.mixed)), flush=True)
+                                   mixed=args.mixed, coordwise=args.coordwise,
+                                   with_q=args.q)), flush=True)
 
 
 if __name__ == "__main__":

@@ -66,7 +66,15 @@ def make_case(K, d, dtype, eta, b_cur, seed, sigma=0.05, noise="normal", shard_o
 
 def run_and_check(K, d, dtype, *, fused, eta=0.1, b_cur=64, seed=1, shard_offsets=None,
                   grad_shift=0, state_shift=0, zero_moments=True, step=1, want_gbar=True,
-                  sigma=0.05):
+                  sigma=0.05, with_q=None):
+    """One call through the C ABI, every output against the oracle.  The unfused test exists
+    with and without the diagnostic Q (abs_norm_test_q / abs_norm_test): with_q=None runs
+    both and returns the results of the one with Q."""
+    if not fused and with_q is None:
+        run_and_check(K, d, dtype, fused=False, eta=eta, b_cur=b_cur, seed=seed,
+                      shard_offsets=shard_offsets, grad_shift=grad_shift, state_shift=state_shift,
+                      sigma=sigma, with_q=False)
+        with_q = True
     grads, ref = make_case(K, d, dtype, eta, b_cur, seed, sigma=sigma, shard_offsets=shard_offsets)
     grads = [shifted_copy(g, grad_shift) for g in grads]
     n_shards = 1 if shard_offsets is None else len(shard_offsets) - 1
@@ -87,17 +95,22 @@ def run_and_check(K, d, dtype, *, fused, eta=0.1, b_cur=64, seed=1, shard_offset
                                  views[0], views[1], views[2], HP, step,
                                  shard_offsets=shard_offsets)
     else:
-        absnt.abs_norm_test(grads, eta, b_cur, stats, gbar, b_next, shard_offsets=shard_offsets)
+        entry = absnt.abs_norm_test_q if with_q else absnt.abs_norm_test
+        entry(grads, eta, b_cur, stats, gbar, b_next, shard_offsets=shard_offsets)
     torch.cuda.synchronize()
     got = absnt.read_stats(stats, n_shards)
 
     assert_sum_close(got["n2"], ref["n2"], "n2")
     assert_sum_close(got["S"], ref["S"], "S")
-    keys = ("n2", "S") if fused else ("n2", "S", "Q")  # the fused kernel leaves Q out (NaN)
-    if fused:
-        assert math.isnan(got["Q"])
-    else:
+    # only abs_norm_test_q computes Q; everywhere else its slots read NaN
+    keys = ("n2", "S", "Q") if with_q else ("n2", "S")
+    if with_q:
         assert_sum_close(got["Q"], ref["Q"], "Q")
+    else:
+        offs_ = shard_offsets if shard_offsets is not None else [0, d]
+        assert math.isnan(got["Q"])
+        for s_, rec in enumerate(got["shards"]):  # an empty shard has nothing to add: 0
+            assert math.isnan(rec[2]) or (offs_[s_ + 1] == offs_[s_] and rec[2] == 0.0)
     assert got["norm"] == K
     assert got["T"] == pytest.approx(ref["T"], rel=3e-6)
     assert int(b_next.item()) == ref["b_next"]
@@ -267,7 +280,7 @@ def test_ragged_shards(dtype):
     got, ref = run_and_check(4, d, dtype, fused=True, seed=700, shard_offsets=offs)
     assert got["shards"][2][:2] == (0.0, 0.0)
     got, ref = run_and_check(4, d, dtype, fused=False, seed=701, shard_offsets=offs)
-    assert got["shards"][2] == (0.0, 0.0, 0.0)
+    assert got["shards"][2] == (0.0, 0.0, 0.0)   # the results of abs_norm_test_q
 
 
 def test_shards_spanning_several_record_slices():
@@ -400,7 +413,7 @@ def test_identical_buffers_keep_batch_size(K, dtype):
     stats = absnt.alloc_stats(d, 1, DEV)
     gbar = torch.empty(d, dtype=torch.float32, device=DEV)
     b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
-    absnt.abs_norm_test(grads, 0.1, 77, stats, gbar, b_next)
+    absnt.abs_norm_test_q(grads, 0.1, 77, stats, gbar, b_next)
     got = absnt.read_stats(stats)
     assert got["S"] == 0.0 and got["T"] == 0.0 and got["flags"] == 0
     assert int(b_next.item()) == 77
@@ -770,11 +783,11 @@ def test_config3_full_size_fsdp_shards():
     got = absnt.read_stats(stats, n_sh)
     dev_b_next = int(b_next.item())
 
-    tot = [0.0, 0.0, 0.0]
+    tot = [0.0, 0.0]
     for s in range(n_sh):
         lo, hi = offs[s], offs[s + 1]
         ref = orc.norm_test([to_host(g[lo:hi]) for g in grads], 0.1, b_cur)
-        for j, key in enumerate(("n2", "S", "Q")):
+        for j, key in enumerate(("n2", "S")):
             assert abs(got["shards"][s][j] - ref[key]) <= 1e-6 * ref[key], (s, key)
             tot[j] += ref[key]  # shard order, as the oracle itself combines shards
         assert_vec_close(gbar[lo:hi], ref["gbar"], "gbar shard %d" % s)
