@@ -60,7 +60,7 @@ typedef enum {
   ABS_ERR_ALIAS = -8   /* an output overlaps a gradient buffer or another output        */
 } abs_status;
 
-enum { ABS_MAX_WORKERS = 64, ABS_MAX_SHARDS = 128 };
+enum { ABS_MAX_WORKERS = 1024, ABS_MAX_SHARDS = 128 };
 
 /* AdamW hyper-parameters (alpha, beta1, beta2, epsilon, lambda of Algorithm 1). */
 typedef struct {
@@ -116,7 +116,9 @@ size_t abs_persample_stats_bytes(int64_t b, int64_t d);
  *
  *   grads          host array of K device pointers, each d elements of `dtype`,
  *                  aligned to the element size (16-byte alignment is faster, not required)
- *   K              1..ABS_MAX_WORKERS
+ *   K              1..ABS_MAX_WORKERS (1024 = 4 workers x 256 accumulation steps, the largest
+ *                  layout of the paper's Table 5, should the J*M micro-batch gradients of a
+ *                  step serve as the samples of the estimator)
  *   d              >= 1
  *   shard_offsets  host array of n_shards+1 non-decreasing offsets, [0]=0, [n_shards]=d;
  *                  NULL = one shard (n_shards ignored)

@@ -19,7 +19,7 @@ ABS_ERR_NULL, ABS_ERR_RANGE, ABS_ERR_SHARDS, ABS_ERR_ALIGN, ABS_ERR_DTYPE, ABS_E
 ABS_ERR_TOO_LARGE = -7
 ABS_ERR_ALIAS = -8
 ABS_NOALLOC_MAX_CHUNKS = 131072
-ABS_MAX_WORKERS, ABS_MAX_SHARDS = 64, 128
+ABS_MAX_WORKERS, ABS_MAX_SHARDS = 1024, 128
 (ABS_STAT_N2, ABS_STAT_S, ABS_STAT_Q, ABS_STAT_T, ABS_STAT_FLAGS, ABS_STAT_NORM,
  ABS_STAT_NCHUNKS, ABS_STAT_ARGMAX) = range(8)
 ABS_STATS_HEADER, ABS_SHARD_STRIDE = 8, 4

@@ -17,7 +17,8 @@ using namespace absnt;
 // The kernels behind these are instantiated in stream_inst.cu, once per combination.
 namespace absnt {
 #define ABS_DECLARE_STREAM(GT, ADAM, STAT) \
-  extern template cudaError_t launch_stream<GT, ADAM, STAT>(const StreamParams&, cudaStream_t);
+  extern template cudaError_t launch_stream<GT, ADAM, STAT>(const StreamParams&, const WideTable*, \
+                                                            cudaStream_t);
 ABS_DECLARE_STREAM(F32, true, kStatSums)
 ABS_DECLARE_STREAM(BF16, true, kStatSums)
 ABS_DECLARE_STREAM(F32, false, kStatSumsQ)
@@ -312,7 +313,15 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
 
   StreamParams prm;
   std::memset(&prm, 0, sizeof prm);
-  for (int k = 0; k < K; ++k) prm.grads[k] = grads[k];
+  WideTable wide_table;  // only filled and passed for more than kInlineWorkers workers
+  const WideTable* wide = nullptr;
+  if (K <= kInlineWorkers) {
+    for (int k = 0; k < K; ++k) prm.grads[k] = grads[k];
+  } else {
+    for (int k = 0; k < K; ++k) wide_table.ptrs[k] = grads[k];
+    for (int k = K; k < ABS_MAX_WORKERS; ++k) wide_table.ptrs[k] = nullptr;
+    wide = &wide_table;
+  }
   std::memcpy(prm.shard_off, L.shard_off, sizeof(int64_t) * (L.n_shards + 1));
   std::memcpy(prm.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
   prm.d = d;
@@ -335,19 +344,19 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   cudaError_t e;
   const bool f32 = dtype == ABS_F32;
   if (stat == kStatCoordwise) {
-    e = fused ? (f32 ? launch_stream<F32, true, kStatCoordwise>(prm, st)
-                     : launch_stream<BF16, true, kStatCoordwise>(prm, st))
-              : (f32 ? launch_stream<F32, false, kStatCoordwise>(prm, st)
-                     : launch_stream<BF16, false, kStatCoordwise>(prm, st));
+    e = fused ? (f32 ? launch_stream<F32, true, kStatCoordwise>(prm, wide, st)
+                     : launch_stream<BF16, true, kStatCoordwise>(prm, wide, st))
+              : (f32 ? launch_stream<F32, false, kStatCoordwise>(prm, wide, st)
+                     : launch_stream<BF16, false, kStatCoordwise>(prm, wide, st));
   } else if (fused) {
-    e = f32 ? launch_stream<F32, true, kStatSums>(prm, st)
-            : launch_stream<BF16, true, kStatSums>(prm, st);
+    e = f32 ? launch_stream<F32, true, kStatSums>(prm, wide, st)
+            : launch_stream<BF16, true, kStatSums>(prm, wide, st);
   } else if (stat == kStatSumsQ) {
-    e = f32 ? launch_stream<F32, false, kStatSumsQ>(prm, st)
-            : launch_stream<BF16, false, kStatSumsQ>(prm, st);
+    e = f32 ? launch_stream<F32, false, kStatSumsQ>(prm, wide, st)
+            : launch_stream<BF16, false, kStatSumsQ>(prm, wide, st);
   } else {
-    e = f32 ? launch_stream<F32, false, kStatSums>(prm, st)
-            : launch_stream<BF16, false, kStatSums>(prm, st);
+    e = f32 ? launch_stream<F32, false, kStatSums>(prm, wide, st)
+            : launch_stream<BF16, false, kStatSums>(prm, wide, st);
   }
   if (e != cudaSuccess) return cuda_fail(e);
 

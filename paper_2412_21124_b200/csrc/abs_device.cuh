@@ -21,9 +21,18 @@ struct AdamScalars {
   float eps, decay;   // epsilon, 1-alpha*lambda
 };
 
+// Up to kInlineWorkers gradient pointers travel inside the parameter block; calls with more
+// workers pass a second kernel parameter, a table of ABS_MAX_WORKERS pointers (8 KB: kernel
+// parameters may be up to 32 KB on this architecture), to a kernel of their own, so that the
+// common launches keep their small parameter block.
+constexpr int kInlineWorkers = 64;
+struct WideTable {
+  const void* ptrs[ABS_MAX_WORKERS];
+};
+
 // Parameter block of the streaming norm-test kernels, passed by value.
 struct StreamParams {
-  const void* grads[ABS_MAX_WORKERS];
+  const void* grads[kInlineWorkers];
   int64_t shard_off[ABS_MAX_SHARDS + 1];    // element offsets of the shards
   int32_t chunk_prefix[ABS_MAX_SHARDS + 1]; // first chunk index of each shard
   int64_t d;

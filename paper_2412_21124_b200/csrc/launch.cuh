@@ -117,8 +117,14 @@ cudaError_t launch_split(const StreamParams& prm, cudaStream_t st) {
 // The fused kernel leaves Q out (its stats slot reads NaN): at the power cap the K extra
 // multiply-adds per coordinate cost about 1% of bandwidth.  The unfused test computes it.
 template <typename GT, bool ADAM, int STAT>
-cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
+cudaError_t launch_stream(const StreamParams& prm, const WideTable* wide, cudaStream_t st) {
   const int K = prm.K;
+  if (K > kInlineWorkers) {
+    // 65..ABS_MAX_WORKERS buffers: the pointer table is a kernel parameter of its own
+    using G4 = typename std::conditional<std::is_same<GT, BF16>::value, BF16H, GT>::type;
+    return launch_pdl(normtest_split_wide_kernel<G4, ADAM, STAT>,
+                      dim3(static_cast<unsigned>(prm.n_chunks)), dim3(kThreads), st, prm, *wide);
+  }
   switch (K) {
     // every count up to 16 has an unrolled kernel of its own (one kernel for a range of counts,
     // predicating the absent workers, ran 10-25% slower: bf16 K=12 5.6 vs 6.9 TB/s, fp32 K=6
@@ -142,7 +148,7 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
     case 32: return launch_split<GT, true, ADAM, STAT>(prm, st);
     case 64:  // bf16: four unrolled groups of 16; fp32 spills in that form and takes the loop
       if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, STAT, 64>(prm, st);
-      else return launch_split<GT, false, ADAM, STAT, ABS_MAX_WORKERS>(prm, st);
+      else return launch_split<GT, false, ADAM, STAT, kInlineWorkers>(prm, st);
     case 17: return launch_split<GT, true, ADAM, STAT, 17>(prm, st);
     case 18: return launch_split<GT, true, ADAM, STAT, 18>(prm, st);
     case 19: return launch_split<GT, true, ADAM, STAT, 19>(prm, st);
@@ -160,11 +166,11 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
     case 31: return launch_split<GT, true, ADAM, STAT, 31>(prm, st);
     case 48:
       if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, STAT, 48>(prm, st);
-      else return launch_split<GT, false, ADAM, STAT, ABS_MAX_WORKERS>(prm, st);
+      else return launch_split<GT, false, ADAM, STAT, kInlineWorkers>(prm, st);
 #define ABS_SPLIT_BF16_CASE(N)                                                              \
   case N:                                                                                   \
     if constexpr (std::is_same<GT, BF16>::value) return launch_split<GT, true, ADAM, STAT, N>(prm, st); \
-    else return launch_split<GT, false, ADAM, STAT, ABS_MAX_WORKERS>(prm, st);
+    else return launch_split<GT, false, ADAM, STAT, kInlineWorkers>(prm, st);
     // the multiples of four above 32 (J workers x M accumulation steps is one in practice)
     ABS_SPLIT_BF16_CASE(36)
     ABS_SPLIT_BF16_CASE(40)
@@ -176,7 +182,7 @@ cudaError_t launch_stream(const StreamParams& prm, cudaStream_t st) {
     default:
       // 33..63 workers without a kernel of their own: run-time groups and unpredicated pieces
       // (5.6-6.1 TB/s; a kernel with compile-time groups runs at 6.4-6.7, as K = 17..32 show)
-      return launch_split<GT, false, ADAM, STAT, ABS_MAX_WORKERS>(prm, st);
+      return launch_split<GT, false, ADAM, STAT, kInlineWorkers>(prm, st);
   }
 }
 

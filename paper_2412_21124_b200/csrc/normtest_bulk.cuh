@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
   bool lost = false;        // a bounded wait ran out
 
   for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
-    const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, K, chunk);
+    const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, prm.grads, K, chunk);
     if (!waited) {  // everything above used kernel parameters only
       grid_dependency_wait();
       waited = true;

@@ -125,6 +125,17 @@ __device__ __forceinline__ float2 coord_math_pair(const float2 (&g)[KB], int K,
   return mean;
 }
 
+// Workers per group of the many-worker kernel: the loads of one group are issued together, and
+// the shifted squares are accumulated per group and the group totals added up.  A flat fp32
+// accumulation over hundreds of workers is biased for bf16 inputs (their squares are short bit
+// patterns that hit rounding ties: S came out 1.4e-6 low at K = 333, 2.5e-6 low at K = 1024);
+// with group totals the error is 3e-8 at K = 1024.  Compile-time worker counts use 16; the
+// run-time loop 16 for bf16 (8-byte vectors) and 8 for fp32.
+template <typename GT, bool EXACT>
+__host__ __device__ constexpr int split_group() {
+  return EXACT ? 16 : (sizeof(typename GT::raw_t) <= 8 ? 16 : 8);
+}
+
 // The same three quantities with the shifted one-pass form used for many workers:
 //   c = g_0;  S_i = sum_k (g_k - c)^2 - K (gbar - c)^2
 // so that the K values need not all be live at once.  The cancellation is bounded: the
@@ -143,17 +154,27 @@ template <typename GT, int KB, bool EXACT, bool WITHQ>
 __device__ __forceinline__ float coord_math_split(const float (&g)[KB], int K,
                                                   const StreamParams& prm, float& dev2, float& sq) {
   constexpr bool kF32Sum = std::is_same<typename GT::sum_t, float>::value;
+  constexpr int H = split_group<GT, EXACT>();
   typename GT::sum_t s = 0;
   const float c = g[0];
-  float s2 = 0.f;
+  float s2 = 0.f, g2 = 0.f;  // total of the closed groups, the open group
+  float gq = 0.f;            // the same for the plain squares
   sq = 0.f;
 #pragma unroll
   for (int k = 0; k < KB; ++k)
     if (EXACT || k < K) {
       s += static_cast<typename GT::sum_t>(g[k]);
       const float dv = g[k] - c;
-      s2 = fmaf(dv, dv, s2);
-      if (WITHQ) sq = fmaf(g[k], g[k], sq);
+      g2 = fmaf(dv, dv, g2);
+      if (WITHQ) gq = fmaf(g[k], g[k], gq);
+      if ((k + 1) % H == 0 || k + 1 == (EXACT ? KB : K)) {
+        s2 += g2;
+        g2 = 0.f;
+        if (WITHQ) {
+          sq += gq;
+          gq = 0.f;
+        }
+      }
     }
   float mean, dm;
   if constexpr (kF32Sum) {
@@ -173,8 +194,8 @@ __device__ __forceinline__ float coord_math_split(const float (&g)[KB], int K,
 // arithmetic in the same order as the vector path, so both give identical bits.  Kept out
 // of line so that its registers do not weigh on the vector path.
 template <typename GT, int KB, bool EXACT, bool ADAM, int STAT, bool SPLIT = false>
-__device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t base, int64_t hi,
-                                        int64_t chunk_lo,
+__device__ __noinline__ void scalar_row(const StreamParams& prm, const void* const* grads, int K,
+                                        int64_t base, int64_t hi, int64_t chunk_lo,
                                         float* sums /* n2, S, Q of this thread-row */,
                                         CwMax* cw) {
   constexpr int V = GT::kVec;
@@ -183,12 +204,48 @@ __device__ __noinline__ void scalar_row(const StreamParams& prm, int K, int64_t 
   for (int e = 0; e < V; ++e) {
     const int64_t i = base + e;
     if (i >= hi) break;  // the remaining coordinates would add exact zeros
-    float g[KB];
+    float dev2, sq, mean;
+    if constexpr (SPLIT && !EXACT) {
+      // any worker count: the arithmetic of coord_math_split with the values consumed as they
+      // are loaded (same operations in the same order)
+      constexpr bool kF32Sum = std::is_same<typename GT::sum_t, float>::value;
+      constexpr int H = split_group<GT, false>();
+      typename GT::sum_t s = 0;
+      const float c = GT::load1(grads[0], i);
+      float s2 = 0.f, g2 = 0.f, gq = 0.f;
+      sq = 0.f;
+      for (int k = 0; k < K; ++k) {
+        const float g = GT::load1(grads[k], i);
+        s += static_cast<typename GT::sum_t>(g);
+        const float dv = g - c;
+        g2 = fmaf(dv, dv, g2);
+        if (WITHQ) gq = fmaf(g, g, gq);
+        if ((k + 1) % H == 0 || k + 1 == K) {
+          s2 += g2;
+          g2 = 0.f;
+          if (WITHQ) {
+            sq += gq;
+            gq = 0.f;
+          }
+        }
+      }
+      float dm;
+      if constexpr (kF32Sum) {
+        mean = mean_of_sum<false>(s, prm.inv_Kf, prm.neg_Kf);
+        dm = fmaf(prm.neg_Kf, c, s) * prm.inv_Kf;
+      } else {
+        const double mx = s * prm.inv_K;
+        mean = static_cast<float>(mx);
+        dm = static_cast<float>(mx - static_cast<double>(c));
+      }
+      dev2 = clamp_nonneg(fmaf(prm.neg_Kf * dm, dm, s2));
+    } else {
+      float g[KB];
 #pragma unroll
-    for (int k = 0; k < KB; ++k) g[k] = (EXACT || k < K) ? GT::load1(prm.grads[k], i) : 0.f;
-    float dev2, sq;
-    const float mean = SPLIT ? coord_math_split<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq)
-                             : coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
+      for (int k = 0; k < KB; ++k) g[k] = (EXACT || k < K) ? GT::load1(grads[k], i) : 0.f;
+      mean = SPLIT ? coord_math_split<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq)
+                   : coord_math<GT, KB, EXACT, WITHQ>(g, K, prm, dev2, sq);
+    }
     row_n2 = fmaf(mean, mean, row_n2);
     row_S += dev2;
     row_Q += sq;
@@ -217,7 +274,9 @@ struct ChunkGeometry {
 };
 
 template <typename GT, int KB, bool EXACT, bool ADAM>
-__device__ __forceinline__ ChunkGeometry chunk_geometry(const StreamParams& prm, int K, int chunk) {
+__device__ __forceinline__ ChunkGeometry chunk_geometry(const StreamParams& prm,
+                                                        const void* const* grads, int K,
+                                                        int chunk) {
   // shard that owns this chunk: largest s with chunk_prefix[s] <= chunk
   int lo_s = 0, hi_s = prm.n_shards;
   while (hi_s - lo_s > 1) {
@@ -230,11 +289,16 @@ __device__ __forceinline__ ChunkGeometry chunk_geometry(const StreamParams& prm,
   const int64_t shard_hi = prm.shard_off[lo_s + 1];
   g.hi = (g.lo + prm.chunk_elems < shard_hi) ? g.lo + prm.chunk_elems : shard_hi;
   uintptr_t bits = 0, bits_f32 = 0;
+  if constexpr (EXACT) {
 #pragma unroll
-  for (int k = 0; k < KB; ++k)
-    if (EXACT || k < K)
-      bits |= reinterpret_cast<uintptr_t>(prm.grads[k]) +
+    for (int k = 0; k < KB; ++k)
+      bits |= reinterpret_cast<uintptr_t>(grads[k]) +
               static_cast<uintptr_t>(g.lo) * sizeof(typename GT::scalar);
+  } else {
+    for (int k = 0; k < K; ++k)
+      bits |= reinterpret_cast<uintptr_t>(grads[k]) +
+              static_cast<uintptr_t>(g.lo) * sizeof(typename GT::scalar);
+  }
   if (prm.gbar) bits_f32 |= reinterpret_cast<uintptr_t>(prm.gbar) + static_cast<uintptr_t>(g.lo) * 4;
   if (ADAM) {
     bits_f32 |= reinterpret_cast<uintptr_t>(prm.p) + static_cast<uintptr_t>(g.lo) * 4;
@@ -431,7 +495,7 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
       }
     } else if (base < hi) {
       float sums[3];
-      scalar_row<GT, KB, EXACT, ADAM, STAT>(prm, K, base, hi, cg.lo, sums, &cw);
+      scalar_row<GT, KB, EXACT, ADAM, STAT>(prm, prm.grads, K, base, hi, cg.lo, sums, &cw);
       row_n2 = sums[0];
       row_S = sums[1];
       row_Q = sums[2];
@@ -490,7 +554,7 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : ((KB <= 16
   const int K = EXACT ? KB : prm.K;
   bool waited = false;
   for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
-    const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, K, chunk);
+    const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, prm.grads, K, chunk);
     if (!waited) {  // everything above used kernel parameters only
       grid_dependency_wait();
       waited = true;
@@ -510,7 +574,8 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : ((KB <= 16
 // CTAs per SM instead of one at 255 registers, and no instructions for absent workers
 // beyond the last group).
 template <typename GT, int KB, bool EXACT, bool ADAM, int STAT>
-__device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
+__device__ __forceinline__ void chunk_rows_split(const StreamParams& prm,
+                                                 const void* const* grads, int K,
                                                  const ChunkGeometry& cg, double& acc_n2,
                                                  double& acc_S, double& acc_Q, CwMax& cw) {
   constexpr int V = GT::kVec;
@@ -521,7 +586,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
   // over groups of 32 bytes
   // per coordinate quad in registers (8 fp32 vectors, 16 bf16 vectors), then the remaining
   // workers in unpredicated pieces of 8, 4, 2 and 1
-  constexpr int H = EXACT ? 16 : (sizeof(typename GT::raw_t) <= 8 ? 16 : 8);
+  constexpr int H = split_group<GT, EXACT>();
   static_assert(EXACT || KB % H == 0, "groups");
   const int tid = threadIdx.x;
   const int64_t hi = cg.hi;
@@ -536,12 +601,23 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
       constexpr int P = V / 2;
       typename GT::sum_t s[V];  // sums of fp32 gradients (fp64)
       float2 sp[P];             // sums of bf16 gradients (fp32, packed)
-      float2 c[P], neg_c[P], s2[P], q[P];
+      float2 c[P], neg_c[P], s2[P], g2[P], q[P], gq[P];  // s2, q: closed groups; g2, gq: the open one
 #pragma unroll
       for (int e = 0; e < V; ++e) s[e] = 0;
 #pragma unroll
       for (int pi = 0; pi < P; ++pi)
-        sp[pi] = c[pi] = neg_c[pi] = s2[pi] = q[pi] = make_float2(0.f, 0.f);
+        sp[pi] = c[pi] = neg_c[pi] = s2[pi] = g2[pi] = q[pi] = gq[pi] = make_float2(0.f, 0.f);
+      auto close_group = [&]() {
+#pragma unroll
+        for (int pi = 0; pi < P; ++pi) {
+          s2[pi] = __fadd2_rn(s2[pi], g2[pi]);
+          g2[pi] = make_float2(0.f, 0.f);
+          if (WITHQ) {
+            q[pi] = __fadd2_rn(q[pi], gq[pi]);
+            gq[pi] = make_float2(0.f, 0.f);
+          }
+        }
+      };
       float4 pw, pm, pv;
       if (ADAM) {  // in flight while the gradients are consumed
         pw = ld_state_16(prm.p + base);
@@ -555,7 +631,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
 #pragma unroll
         for (int k = 0; k < N; ++k)
           raw[k] = GT::load_vec(
-              reinterpret_cast<const typename GT::scalar*>(prm.grads[k0 + k]) + base);
+              reinterpret_cast<const typename GT::scalar*>(grads[k0 + k]) + base);
 #pragma unroll
         for (int pi = 0; pi < P; ++pi) {
 #pragma unroll
@@ -572,21 +648,31 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
               s[2 * pi] += static_cast<typename GT::sum_t>(g.x);
               s[2 * pi + 1] += static_cast<typename GT::sum_t>(g.y);
             }
-            s2[pi] = __ffma2_rn(dv, dv, s2[pi]);
-            if (WITHQ) q[pi] = __ffma2_rn(g, g, q[pi]);
+            g2[pi] = __ffma2_rn(dv, dv, g2[pi]);
+            if (WITHQ) gq[pi] = __ffma2_rn(g, g, gq[pi]);
           }
         }
       };
       if constexpr (EXACT) {
 #pragma unroll
-        for (int h = 0; h < KB / H; ++h) group(h * H, std::integral_constant<int, H>{});
-        if constexpr (KB % H != 0) group(KB / H * H, std::integral_constant<int, KB % H>{});
+        for (int h = 0; h < KB / H; ++h) {
+          group(h * H, std::integral_constant<int, H>{});
+          close_group();
+        }
+        if constexpr (KB % H != 0) {
+          group(KB / H * H, std::integral_constant<int, KB % H>{});
+          close_group();
+        }
       } else {
         // whole groups in a run-time loop, then the remainder in pieces of 8, 4, 2, 1 workers:
         // no load is predicated on the worker count
         int k0 = 0;
 #pragma unroll 1
-        for (; k0 + H <= K; k0 += H) group(k0, std::integral_constant<int, H>{});
+        for (; k0 + H <= K; k0 += H) {
+          group(k0, std::integral_constant<int, H>{});
+          close_group();
+        }
+        // the rest (fewer than H workers) is one more group, taken in pieces
         if (H > 8 && ((K - k0) & 8)) {
           group(k0, std::integral_constant<int, 8>{});
           k0 += 8;
@@ -600,6 +686,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
           k0 += 2;
         }
         if ((K - k0) & 1) group(k0, std::integral_constant<int, 1>{});
+        close_group();  // adds exact zeros when K is a multiple of H
       }
       float gb[V];
       float2* w2 = reinterpret_cast<float2*>(&pw);
@@ -644,7 +731,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm, int K,
       }
     } else if (base < hi) {
       float sums[3];
-      scalar_row<GT, KB, EXACT, ADAM, STAT, true>(prm, K, base, hi, cg.lo, sums, &cw);
+      scalar_row<GT, KB, EXACT, ADAM, STAT, true>(prm, grads, K, base, hi, cg.lo, sums, &cw);
       row_n2 = sums[0];
       row_S = sums[1];
       row_Q = sums[2];
@@ -662,7 +749,7 @@ __global__ void __launch_bounds__(kThreads, 2)
   const int K = EXACT ? KB : prm.K;
   bool waited = false;
   for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
-    const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, K, chunk);
+    const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, prm.grads, K, chunk);
     if (!waited) {
       grid_dependency_wait();
       waited = true;
@@ -670,7 +757,7 @@ __global__ void __launch_bounds__(kThreads, 2)
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
     CwMax cw;
     cw.init(static_cast<int>(threadIdx.x) * GT::kVec);
-    chunk_rows_split<GT, KB, EXACT, ADAM, STAT>(prm, K, cg, acc_n2, acc_S, acc_Q, cw);
+    chunk_rows_split<GT, KB, EXACT, ADAM, STAT>(prm, prm.grads, K, cg, acc_n2, acc_S, acc_Q, cw);
     write_chunk_record<STAT>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, cw, red);
   }
 }
@@ -694,6 +781,31 @@ constexpr int kFinalizeMaxCtas = 8;
 constexpr int kFinalizeSlice = 128;       // records: 32 lanes x 4 loads in flight
 constexpr int kFinalizeMaxSlices = 1024;  // 24 KB of partials in CTA 0
 constexpr int kFinalizeSlicesPerCta = 16;  // another CTA (another SM's L2 port) per 16 slices
+
+// More than kInlineWorkers workers (up to ABS_MAX_WORKERS): the run-time loop of the kernel
+// above over a pointer table that arrives as a second kernel parameter.
+template <typename GT, bool ADAM, int STAT>
+__global__ void __launch_bounds__(kThreads, 2)
+    normtest_split_wide_kernel(const __grid_constant__ StreamParams prm,
+                               const __grid_constant__ WideTable table) {
+  __shared__ double red[kWarps * 3];
+  const int K = prm.K;
+  bool waited = false;
+  for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
+    const ChunkGeometry cg =
+        chunk_geometry<GT, kInlineWorkers, false, ADAM>(prm, table.ptrs, K, chunk);
+    if (!waited) {
+      grid_dependency_wait();
+      waited = true;
+    }
+    double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
+    CwMax cw;
+    cw.init(static_cast<int>(threadIdx.x) * GT::kVec);
+    chunk_rows_split<GT, kInlineWorkers, false, ADAM, STAT>(prm, table.ptrs, K, cg, acc_n2, acc_S,
+                                                            acc_Q, cw);
+    write_chunk_record<STAT>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, cw, red);
+  }
+}
 
 // records c0 + first, c0 + first + stride, ... (< c1), added in that order.  Each pass issues
 // four unconditional loads (an index past the end re-reads the pass's first record and its

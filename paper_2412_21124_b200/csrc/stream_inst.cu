@@ -16,5 +16,5 @@
 
 namespace absnt {
 template cudaError_t launch_stream<ABS_INST_GT, ABS_INST_ADAM != 0, ABS_INST_STAT>(
-    const StreamParams&, cudaStream_t);
+    const StreamParams&, const WideTable*, cudaStream_t);
 }  // namespace absnt

@@ -241,7 +241,7 @@ def _offs(*vals):
     (dict(b_next=None), binding.ABS_ERR_NULL),
     (dict(dtype=2), binding.ABS_ERR_DTYPE),
     (dict(K=0), binding.ABS_ERR_RANGE),
-    (dict(K=65), binding.ABS_ERR_RANGE),
+    (dict(K=binding.ABS_MAX_WORKERS + 1), binding.ABS_ERR_RANGE),
     (dict(d=0), binding.ABS_ERR_RANGE),
     (dict(b_cur=0), binding.ABS_ERR_RANGE),
     (dict(eta=0.0), binding.ABS_ERR_RANGE),

@@ -45,7 +45,8 @@ def _device():
 #   16  fused bf16: bulk, 512 tile; fused fp32: register-direct
 #   24, 32   many-worker kernel, compile-time groups
 #   33, 47   many-worker kernel, run-time groups
-FAMILY_K = [2, 4, 8, 12, 16, 24, 32, 33, 47]
+#   100      the same with the pointer table as a kernel parameter of its own (K > 64)
+FAMILY_K = [2, 4, 8, 12, 16, 24, 32, 33, 47, 100]
 # four full 4096-coordinate chunks (staged path where the kernel has one) and a ragged fifth
 # chunk that ends in a partial thread-row (register-direct and element-wise paths)
 D_EDGE = 4 * 4096 + 1234

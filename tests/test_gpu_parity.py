@@ -231,6 +231,20 @@ def test_more_than_32_workers(K, dtype):
                   grad_shift=1 if K == 48 else 0)
 
 
+@pytest.mark.parametrize("K,dtype", [(65, torch.bfloat16), (65, torch.float32), (100, torch.bfloat16),
+                                     (128, torch.float32), (333, torch.bfloat16),
+                                     (1024, torch.bfloat16), (1024, torch.float32)],
+                         ids=lambda x: str(x).replace("torch.", ""))
+def test_more_than_64_workers(K, dtype):
+    """65..1024 buffers (4 workers x 256 accumulation steps is the largest layout of the paper's
+    Table 5): the pointer table travels as a kernel parameter of its own."""
+    d = 2 * 4096 + 1_234 if K <= 333 else 4096 + 321
+    run_and_check(K, d, dtype, fused=True, seed=580 + K, zero_moments=False, step=3)
+    run_and_check(K, d, dtype, fused=True, seed=581 + K, zero_moments=True, step=1,
+                  grad_shift=1, state_shift=3)
+    run_and_check(K, d, dtype, fused=False, seed=582 + K, shard_offsets=[0, 5, 4101, d])
+
+
 def _random_case(i):
     rng = np.random.default_rng(9000 + i)
     K = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 11, 13, 16, 17, 23, 24, 31, 32, 33, 47, 48, 63, 64]))
