@@ -100,7 +100,7 @@ enum {
 size_t abs_stats_bytes(int64_t d, int n_shards);
 
 /* Bytes the caller must provide for stats_out of abs_persample_norm_test (b rows of d
- * columns): header + one shard record + chunk scratch + the row-block work space.
+ * columns): header + one shard record + the row-block work space + its ticket counters.
  * Returns 0 on invalid arguments.  Host, pure.                                          */
 size_t abs_persample_stats_bytes(int64_t b, int64_t d);
 
@@ -275,13 +275,20 @@ int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64_t d, abs_d
 /*
  * Approximate norm test on per-sample gradients (Eq. 3, the Var definition before it,
  * and the b_{k+1} display after it) -- the single-device form of the test.
- *   G          device, row-major [b, ld]; row i = gradient of sample i; read once
+ *   G          device, row-major [b, ld] elements of `dtype`; row i = gradient of sample i;
+ *              read once.  Rows that start on a 16-byte (fp32) / 8-byte (bf16) boundary take
+ *              the fast path; any element-aligned matrix is accepted
  *   b          >= 2 rows (also the current batch size), d >= 1 columns, ld >= d
- *   dtype      ABS_F32 (ABS_BF16 is rejected with ABS_ERR_DTYPE)
+ *   dtype      ABS_F32 or ABS_BF16 (Sec. 5: the experiments train in bfloat16)
  *   gbar[c] = (1/b) sum_i G[i,c];  S = sum_i ||G[i,:]-gbar||^2;  ||Var||_1 = S/(b-1)
  *   T = ||Var||_1 / (eta^2 ||gbar||^2);  b_next = ceil(T) if T > b else b
  *   stats_out  device, abs_persample_stats_bytes(b, d) bytes, 16-byte aligned; header
- *              as above with NORM = b-1 and one shard record
+ *              as above with NORM = b-1 and one shard record; the diagnostic Q is not
+ *              computed (NaN).  The buffer must be ZERO-FILLED before its first use with
+ *              this call (for a given b, d): the thread blocks of its last kernel count
+ *              themselves off in a ticket counter kept in this buffer; the counter is back
+ *              at zero when the call completes, so the buffer can be reused as it is.  Zero it again after a call that returned ABS_ERR_CUDA, or
+ *              before using it with another (b, d).
  *   gbar_out   device, d floats;  b_next_out device, one int64
  */
 int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs_dtype dtype,

@@ -208,10 +208,11 @@ def alloc_stats(d, n_shards=1, device="cuda"):
 
 
 def alloc_persample_stats(b, d, device="cuda"):
+    """A zero-filled stats_out for abs_persample_norm_test (its ticket counters start at 0)."""
     nbytes = abs_persample_stats_bytes(b, d)
     if nbytes == 0:
         raise ValueError("invalid (b, d)")
-    return torch.empty(nbytes // 8, dtype=torch.float64, device=device)
+    return torch.zeros(nbytes // 8, dtype=torch.float64, device=device)
 
 
 # ------------------------------------------------------------------------- entry points

@@ -378,13 +378,15 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
 }
 
 // Rows per row block of the per-sample kernels: at most 512 (the row-block records then cost
-// 2% of the matrix traffic), and, while the grid is only a few waves of 148 SMs x 3 resident
+// 1.6% of the matrix traffic), and, while the grid is only a few waves of 148 SMs x 3 resident
 // CTAs, the count that fills whole waves (b=4096, d=16384: 13 row blocks x 32 column blocks =
-// 416 CTAs in one wave instead of 1024 in 2.3).  A function of (b, d) alone, so the shape of
+// 416 of 444 CTA slots in one wave).  A function of (b, d) alone, so the shape of
 // every sum is too.
+int64_t persample_col_blocks(int64_t d) { return ((d + 3) / 4 + kPsThreads - 1) / kPsThreads; }
+
 int persample_rows_per_block(int64_t b, int64_t d) {
-  const int64_t wave = 148 * 3;
-  const int64_t col_blocks = ((d + 3) / 4 + kPsThreads - 1) / kPsThreads;
+  const int64_t wave = 148 * kPsCtasPerSM;
+  const int64_t col_blocks = persample_col_blocks(d);
   const int64_t nrb_min = (b + 511) / 512;
   int64_t nrb = nrb_min;
   if (nrb_min * col_blocks < 4 * wave) {
@@ -417,11 +419,12 @@ size_t abs_stats_bytes(int64_t d, int n_shards) {
 size_t abs_persample_stats_bytes(int64_t b, int64_t d) {
   if (b < 2 || d < 1) return 0;
   const int rpb = persample_rows_per_block(b, d);
-  const int64_t nrb = (b + rpb - 1) / rpb;
-  const int64_t n_chunks = (d + kPsThreads - 1) / kPsThreads;
-  return sizeof(double) *
-         (ABS_STATS_HEADER + ABS_SHARD_STRIDE + static_cast<size_t>(n_chunks) * 4 +
-          3 * static_cast<size_t>(nrb) * static_cast<size_t>(d));
+  const size_t nrb = static_cast<size_t>((b + rpb - 1) / rpb);
+  const size_t nmb = static_cast<size_t>((d + kPsThreads - 1) / kPsThreads);
+  // header, one shard record, {n2, S} per CTA of the merge pass, {sum, M2} per (row block,
+  // column), and the ticket counter (one double's worth)
+  return sizeof(double) * (ABS_STATS_HEADER + ABS_SHARD_STRIDE + 2 * nmb +
+                           2 * nrb * static_cast<size_t>(d) + 1);
 }
 
 int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
@@ -547,67 +550,60 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
                             double eta, void* stats_out, float* gbar_out, int64_t* b_next_out,
                             abs_stream_t stream) {
   if (!G || !stats_out || !gbar_out || !b_next_out) return ABS_ERR_NULL;
-  if (dtype != ABS_F32) return ABS_ERR_DTYPE;
+  if (dtype != ABS_F32 && dtype != ABS_BF16) return ABS_ERR_DTYPE;
   if (b < 2 || d < 1 || ld < d) return ABS_ERR_RANGE;
   if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
-  if (misaligned(G, 4) || misaligned(gbar_out, 4) || misaligned(stats_out, 16) ||
+  const size_t esz = (dtype == ABS_F32) ? 4 : 2;
+  if (misaligned(G, esz) || misaligned(gbar_out, 4) || misaligned(stats_out, 16) ||
       misaligned(b_next_out, 8))
     return ABS_ERR_ALIGN;
-  const int64_t n_chunks64 = (d + kPsThreads - 1) / kPsThreads;
+  const int64_t ncb = persample_col_blocks(d);
   const int rpb = persample_rows_per_block(b, d);
   const int64_t nrb = (b + rpb - 1) / rpb;
-  if (n_chunks64 > INT32_MAX || nrb > 65535) return ABS_ERR_RANGE;
-
-  if (overlaps(G, static_cast<size_t>(b - 1) * ld * 4 + static_cast<size_t>(d) * 4, gbar_out,
+  if (ncb > INT32_MAX || nrb > 65535) return ABS_ERR_RANGE;
+  if (overlaps(G, (static_cast<size_t>(b - 1) * ld + static_cast<size_t>(d)) * esz, gbar_out,
                static_cast<size_t>(d) * 4))
     return ABS_ERR_ALIAS;
-  const int finalize_ctas = finalize_max_cluster();
 
   double* stats = static_cast<double*>(stats_out);
   PersampleParams prm;
   std::memset(&prm, 0, sizeof prm);
-  prm.G = static_cast<const float*>(G);
+  prm.G = G;
   prm.b = b;
   prm.d = d;
   prm.ld = ld;
   prm.rows_per_block = rpb;
   prm.n_row_blocks = static_cast<int>(nrb);
-  prm.chunk_out = stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE;
-  prm.ws_mean = prm.chunk_out + n_chunks64 * 4;
-  prm.ws_m2 = prm.ws_mean + nrb * d;
-  prm.ws_q = prm.ws_m2 + nrb * d;
+  const int64_t nmb = (d + kPsThreads - 1) / kPsThreads;  // CTAs of the merge pass
+  if (nmb > INT32_MAX) return ABS_ERR_RANGE;
+  prm.cb_rec = stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE;
+  prm.ws_sum = prm.cb_rec + 2 * nmb;
+  prm.ws_m2 = prm.ws_sum + nrb * d;
+  prm.tickets = reinterpret_cast<unsigned int*>(prm.ws_m2 + nrb * d);
   prm.gbar = gbar_out;
+  prm.stats = stats;
+  prm.b_next = b_next_out;
+  prm.eta = eta;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const bool vec = !misaligned(G, 16) && (ld % 4 == 0);
+  // rows that start on a vector boundary (16 bytes of fp32, 8 of bf16) go through the
+  // asynchronous-copy ring; anything else takes element loads with the same arithmetic
+  const size_t vec_bytes = 4 * esz;
+  const bool ring = !misaligned(G, vec_bytes) && ((ld * esz) % vec_bytes == 0);
+  const dim3 grid(static_cast<unsigned>(ncb), static_cast<unsigned>(nrb));
+  const size_t ring_bytes = static_cast<size_t>(kRing) * kPsThreads * vec_bytes;
   cudaError_t e;
-  if (vec) {
-    const int64_t cols = (d + 3) / 4;
-    dim3 grid(static_cast<unsigned>((cols + kPsThreads - 1) / kPsThreads),
-              static_cast<unsigned>(nrb));
-    e = launch_pdl(persample_partial_kernel<4>, grid, dim3(kPsThreads), st, prm);
-  } else {
-    dim3 grid(static_cast<unsigned>(n_chunks64), static_cast<unsigned>(nrb));
-    e = launch_pdl(persample_partial_kernel<1>, grid, dim3(kPsThreads), st, prm);
-  }
+  if (dtype == ABS_F32)
+    e = ring ? launch_pdl_smem(persample_partial_kernel<PsF32, true>, grid, dim3(kPsThreads), ring_bytes,
+                               st, prm)
+             : launch_pdl(persample_partial_kernel<PsF32, false>, grid, dim3(kPsThreads), st, prm);
+  else
+    e = ring ? launch_pdl_smem(persample_partial_kernel<PsBF16, true>, grid, dim3(kPsThreads), ring_bytes,
+                               st, prm)
+             : launch_pdl(persample_partial_kernel<PsBF16, false>, grid, dim3(kPsThreads), st, prm);
   if (e != cudaSuccess) return cuda_fail(e);
-  e = launch_pdl(persample_merge_kernel, dim3(static_cast<unsigned>(n_chunks64)), dim3(kPsThreads),
-                 st, prm);
-  if (e != cudaSuccess) return cuda_fail(e);
-
-  FinalizeParams fp;
-  std::memset(&fp, 0, sizeof fp);
-  fp.chunk_in = prm.chunk_out;
-  fp.chunk_prefix[0] = 0;
-  fp.chunk_prefix[1] = static_cast<int32_t>(n_chunks64);
-  fp.n_shards = 1;
-  fp.n_chunks = static_cast<int>(n_chunks64);
-  fp.stats = stats;
-  fp.b_next = b_next_out;
-  fp.eta = eta;
-  fp.norm = static_cast<double>(b - 1);
-  fp.b_cur = b;
-  e = launch_finalize(fp, finalize_ctas, st);
+  e = launch_pdl(persample_merge_kernel, dim3(static_cast<unsigned>(nmb)), dim3(kPsThreads), st,
+                 prm);
   if (e != cudaSuccess) return cuda_fail(e);
   return ABS_OK;
 }

@@ -14,7 +14,7 @@ Timing: CUDA events on the launching stream around `steps` back-to-back calls af
 replays are timed, so that the figure is device time.  Points whose working set is smaller than twice the L2 rotate over several
 independent buffer sets so that every call reads cold data.  GB/s counts algorithmic bytes:
 fused (K*s + 24) per coordinate (+4 with --gbar, +2 with --mixed), normtest K*s + 4,
-adamw 28 (+2 with --mixed), persample 4 per matrix element.
+adamw 28 (+2 with --mixed), persample 4 (fp32) or 2 (bf16) per matrix element.
 """
 import argparse
 import json
@@ -48,7 +48,7 @@ def bytes_per_call(call, d, K, esz, gbar, b):
         return (K * esz + 4) * d
     if call == "adamw":
         return 28 * d
-    return 4 * b * d
+    return esz * b * d
 
 
 def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b=4096, dev="cuda",
@@ -77,7 +77,7 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
             if call == "adamw":
                 s["gbar"].normal_().mul_(0.02)
         if call == "persample":
-            s["G"] = torch.empty(b, d, dtype=torch.float32, device=dev).normal_().mul_(0.3)
+            s["G"] = torch.empty(b, d, dtype=torch.float32, device=dev).normal_().mul_(0.3).to(tdt)
             s["stats"] = B.alloc_persample_stats(b, d, dev)
             s["gbar"] = torch.zeros(d, dtype=torch.float32, device=dev)
         s["b_next"] = torch.zeros(1, dtype=torch.int64, device=dev)
@@ -180,7 +180,8 @@ REPORT_POINTS = (
     + [("adamw", GPT2, 0, "f32", 1, {}), ("adamw", LLAMA, 0, "f32", 1, {}),
        ("adamw", GPT2, 0, "f32", 1, {"mixed": True})]
     + [("persample", 16_384, 0, "f32", 1, {"b": b}) for b in (4096, 1024, 256, 32)]
-    + [("persample", 65_536, 0, "f32", 1, {"b": 4096})]
+    + [("persample", 65_536, 0, "f32", 1, {"b": 4096}), ("persample", 16_384, 0, "bf16", 1, {"b": 4096}),
+       ("persample", 65_536, 0, "bf16", 1, {"b": 8192})]
     + [("fused", GPT2, 8, "bf16", 1, {"gbar": True}), ("fused", GPT2, 8, "bf16", 1, {"mixed": True}),
        ("fused", 1_048_576, 4, "f32", 1, {})]
     + [("fused", GPT2, K, "bf16", 1, {}) for K in (6, 12, 20, 24, 27, 31, 36, 40, 44, 48, 52, 56,

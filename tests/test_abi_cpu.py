@@ -212,8 +212,8 @@ def test_stats_bytes(L):
     big = binding.abs_stats_bytes(124_439_808, 8)
     assert big % 16 == 0 and big < (1 << 20)
     assert binding.abs_persample_stats_bytes(1, 10) == 0
-    # three doubles per (row block, column), row blocks of at most 512 rows
-    assert binding.abs_persample_stats_bytes(4096, 16384) > 3 * (4096 // 512) * 16384 * 8
+    # two doubles per (row block, column), row blocks of at most 512 rows
+    assert binding.abs_persample_stats_bytes(4096, 16384) > 2 * (4096 // 512) * 16384 * 8
 
 
 # ---- invalid arguments: every path returns its status before any CUDA call ---------------
@@ -333,7 +333,8 @@ def test_adamw_rejects_pointers(L):
 @pytest.mark.parametrize("args,status", [
     ((None, 4, 10, 10, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_NULL),
     ((FAKE, 4, 10, 10, 0, 0.1, None, FAKE, FAKE, None), binding.ABS_ERR_NULL),
-    ((FAKE, 4, 10, 10, 1, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_DTYPE),
+    ((FAKE, 4, 10, 10, 2, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_DTYPE),
+    ((FAKE + 1, 4, 10, 10, 1, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_ALIGN),
     ((FAKE, 1, 10, 10, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_RANGE),
     ((FAKE, 4, 0, 10, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_RANGE),
     ((FAKE, 4, 10, 9, 0, 0.1, FAKE, FAKE, FAKE, None), binding.ABS_ERR_RANGE),
