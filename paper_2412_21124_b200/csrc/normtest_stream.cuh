@@ -6,8 +6,10 @@
 // chunk, row r assigns the V = 16/sizeof(grad) consecutive coordinates starting at
 // chunk_lo + (r*kThreads + tid)*V to thread tid, so the coordinate -> thread -> partial
 // sum mapping depends only on (shard offsets, chunk_elems), never on the grid.  One
-// {n2, S, Q} triple per chunk goes to scratch; the finalize kernel adds chunk triples in
-// a fixed order per shard and shard records in shard order.
+// record per chunk goes to scratch -- {n2, S, Q} (Q only in the diagnostic mode, else NaN), or
+// {n2, S, index, ratio} of the chunk's largest per-coordinate ratio in the coordinate-wise
+// mode; the finalize kernel combines chunk records in a fixed order per shard and shard
+// records in shard order.
 //
 // Per coordinate (Algorithm 1, "Compute the batch gradient" .. "approximate gradient
 // variance"): gbar = fp32(sum_k g_k / K).  fp32 inputs are summed in fp64, so gbar is the
@@ -15,7 +17,7 @@
 // k = 0..K-1 in order: every partial sum is exact unless the addends' exponents spread
 // over more than 13 binades (8-bit significands in a 24-bit accumulator), and fp64
 // conversions would cost ~3% of bandwidth at the power cap.  Deviations g_k - gbar and
-// their squares (and, in the unfused kernel, g_k^2) are fp32 over at most V*K terms per
+// their squares (and, in the diagnostic mode, g_k^2) are fp32 over at most V*K terms per
 // thread-row, then accumulated in fp64.  The fused kernels and the many-worker kernel do
 // this arithmetic two adjacent coordinates at a time with the packed fp32 instructions of
 // sm_100 (coord_math_pair, adamw_pair); every lane rounds like the scalar instruction, so
