@@ -172,6 +172,25 @@ int abs_adamw_step_clipped(float* params, const float* gbar, float* m, float* v,
                            const void* stats_in, abs_stream_t stream);
 
 /*
+ * The fused step with the gradient clipped by the PREVIOUS step's global norm -- a single-pass
+ * approximation of abs_norm_test + abs_adamw_step_clipped (40 instead of 48 B per coordinate at
+ * K = 8 bf16).  It is NOT what the paper's experiments compute: they clip by the norm of the
+ * gradient being applied, which is only known once the whole vector has been read; here
+ *   scale = min(1, max_norm / (sqrt(n2_prev) + 1e-6)),  AdamW on scale * gbar,
+ * with n2_prev = ||gbar||^2 of the step before, read on the device from `stats_prev` -- the
+ * stats_out of the previous call.  stats_prev may be the very buffer passed as stats_out (its
+ * header is read before this call's last kernel rewrites it); NULL = no clipping (the first
+ * step).  The test's statistics and gbar_out are those of the unclipped gradient.  All other
+ * arguments as abs_normtest_adamw; max_norm finite and > 0 when stats_prev is given.
+ */
+int abs_normtest_adamw_clip_prev(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                                 const int64_t* shard_offsets, int n_shards, double eta,
+                                 int64_t b_cur, void* stats_out, float* gbar_out,
+                                 int64_t* b_next_out, float* params, float* m, float* v,
+                                 const abs_adamw_hparams* hparams, int64_t step, double max_norm,
+                                 const void* stats_prev, abs_stream_t stream);
+
+/*
  * The fused step: abs_norm_test and abs_adamw_step in one pass, so gradients and
  * optimizer state cross HBM once.  Arguments as above; gbar_out may be NULL (the mean
  * then lives only in registers).  The diagnostic Q is not computed here: its slots in

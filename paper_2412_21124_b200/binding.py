@@ -72,6 +72,9 @@ def lib():
                                      ptr, ptr, ptr, ptr, i64, ptr]
     L.abs_normtest_adamw_noalloc.restype = cint
     L.abs_normtest_adamw_noalloc.argtypes = list(L.abs_normtest_adamw.argtypes)
+    L.abs_normtest_adamw_clip_prev.restype = cint
+    L.abs_normtest_adamw_clip_prev.argtypes = [ptr, cint, i64, cint, ptr, cint, dbl, i64, ptr, ptr,
+                                               ptr, ptr, ptr, ptr, ptr, i64, dbl, ptr, ptr]
     L.abs_norm_test_coordwise.restype = cint
     L.abs_norm_test_coordwise.argtypes = list(L.abs_norm_test.argtypes)
     L.abs_norm_test_q.restype = cint
@@ -299,6 +302,34 @@ def abs_normtest_adamw_coordwise(grads, eta, b_cur, stats_out, gbar_out, b_next_
     """The fused step with the coordinate-wise test as its decision."""
     abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v, hparams,
                        step, shard_offsets, stream, _entry="abs_normtest_adamw_coordwise")
+
+
+def abs_normtest_adamw_clip_prev(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v,
+                                 hparams, step, max_norm, stats_prev, shard_offsets=None,
+                                 stream=None):
+    """The fused step with the gradient clipped by the previous step's global norm, read on the
+    device from `stats_prev` (the previous call's stats_out; may be `stats_out` itself; None =
+    no clipping).  A single-pass approximation, not what the paper's experiments compute."""
+    table, K, d, code = _grad_table(grads)
+    offs, n_shards = _offsets(shard_offsets)
+    for t, name in ((params, "params"), (m, "m"), (v, "v")):
+        _check_f32_vec(t, d, name)
+    if gbar_out is not None:
+        _check_f32_vec(gbar_out, d, "gbar_out")
+    _check_stats(stats_out, abs_stats_bytes(d, n_shards))
+    if stats_prev is not None:
+        _check_stats(stats_prev, 8 * ABS_STATS_HEADER, "stats_prev")
+    _check_b_next(b_next_out)
+    _check_one_device(*grads, stats_out, gbar_out, b_next_out, params, m, v, stats_prev)
+    hp = _hparams(hparams)
+    rc = lib().abs_normtest_adamw_clip_prev(
+        table, K, d, code, offs, n_shards, float(eta), int(b_cur), stats_out.data_ptr(),
+        gbar_out.data_ptr() if gbar_out is not None else None, b_next_out.data_ptr(),
+        params.data_ptr(), m.data_ptr(), v.data_ptr(), ctypes.byref(hp), int(step),
+        float(max_norm), stats_prev.data_ptr() if stats_prev is not None else None,
+        _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_normtest_adamw_clip_prev")
 
 
 def _check_bf16_vec(t, d, name):

@@ -261,7 +261,7 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                   void* stats_out, float* gbar_out, int64_t* b_next_out, float* params, float* m,
                   float* v, void* params_bf16, const abs_adamw_hparams* hparams, int64_t step,
                   bool fused, abs_stream_t stream, bool builtin_records = false,
-                  int stat = -1) {
+                  int stat = -1, const double* clip_n2 = nullptr, double clip_max_norm = 0.0) {
   if (stat < 0) stat = kStatSums;
   if (!grads || !stats_out || !b_next_out) return ABS_ERR_NULL;
   if (!fused && !gbar_out) return ABS_ERR_NULL;
@@ -338,6 +338,8 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   prm.v = v;
   prm.p16 = static_cast<uint16_t*>(params_bf16);
   prm.chunk_out = chunk_out;
+  prm.clip_n2 = clip_n2;
+  prm.clip_max_norm = clip_max_norm;
   if (fused) prm.adam = make_adam(hparams, step);
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -481,6 +483,23 @@ int abs_normtest_adamw_coordwise(const void* const* grads, int K, int64_t d, abs
   return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
                        gbar_out, b_next_out, params, m, v, nullptr, hparams, step, true, stream,
                        false, kStatCoordwise);
+}
+
+int abs_normtest_adamw_clip_prev(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                                 const int64_t* shard_offsets, int n_shards, double eta,
+                                 int64_t b_cur, void* stats_out, float* gbar_out,
+                                 int64_t* b_next_out, float* params, float* m, float* v,
+                                 const abs_adamw_hparams* hparams, int64_t step, double max_norm,
+                                 const void* stats_prev, abs_stream_t stream) {
+  const double* n2_prev = nullptr;
+  if (stats_prev) {
+    if (!std::isfinite(max_norm) || !(max_norm > 0.0)) return ABS_ERR_RANGE;
+    if (misaligned(stats_prev, 8)) return ABS_ERR_ALIGN;
+    n2_prev = static_cast<const double*>(stats_prev) + ABS_STAT_N2;
+  }
+  return run_norm_test(grads, K, d, dtype, shard_offsets, n_shards, eta, b_cur, stats_out,
+                       gbar_out, b_next_out, params, m, v, nullptr, hparams, step, true, stream,
+                       false, kStatSums, n2_prev, max_norm);
 }
 
 namespace {

@@ -47,6 +47,10 @@ struct StreamParams {
   float* m;
   float* v;
   uint16_t* p16; // fused AdamW, mixed precision: bf16 copy of the updated parameters, may be null
+  // fused AdamW with the gradient clipped by a norm known before the pass (the previous
+  // step's ||gbar||^2, read on the device): null = no clipping
+  const double* clip_n2;
+  double clip_max_norm;
   double* chunk_out; // 4 doubles per chunk: n2, S, Q, 0
   AdamScalars adam;
 };
@@ -145,10 +149,13 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // -- this kernel runs at the board's power cap, where instructions saved are bandwidth
 // gained.  Flushing only matters for vhat below 1.2e-38 (its root is then below 1.1e-19
 // and vanishes against any practical eps).
-__device__ __forceinline__ void adamw_elem(const AdamScalars& a, float g, float& w, float& m,
-                                           float& v) {
-  m = fmaf(a.beta1, m, a.omb1 * g);
-  v = fmaf(a.beta2, v, (a.omb2 * g) * g);
+// omb1, omb2: (1-beta1) and (1-beta2), or those times s and s^2 when the gradient is clipped
+// by a scale s known before the pass (GradWeights below) -- clipping then costs no instruction
+// per coordinate.
+__device__ __forceinline__ void adamw_elem(const AdamScalars& a, float omb1, float omb2, float g,
+                                           float& w, float& m, float& v) {
+  m = fmaf(a.beta1, m, omb1 * g);
+  v = fmaf(a.beta2, v, (omb2 * g) * g);
   float root, inv;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root) : "f"(v * a.inv_bc2));
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(root + a.eps));
@@ -158,11 +165,11 @@ __device__ __forceinline__ void adamw_elem(const AdamScalars& a, float g, float&
 // The same update for two adjacent coordinates with the packed fp32 instructions of sm_100
 // (fma/add/mul.f32x2: one issue slot for both lanes, each lane rounded exactly like the
 // scalar instruction, so the results are bit-identical to two adamw_elem calls).
-__device__ __forceinline__ void adamw_pair(const AdamScalars& a, float2 g, float2& w, float2& m,
-                                           float2& v) {
+__device__ __forceinline__ void adamw_pair(const AdamScalars& a, float omb1, float omb2, float2 g,
+                                           float2& w, float2& m, float2& v) {
   const float2 b1 = make_float2(a.beta1, a.beta1), b2 = make_float2(a.beta2, a.beta2);
-  m = __ffma2_rn(b1, m, __fmul2_rn(make_float2(a.omb1, a.omb1), g));
-  v = __ffma2_rn(b2, v, __fmul2_rn(__fmul2_rn(make_float2(a.omb2, a.omb2), g), g));
+  m = __ffma2_rn(b1, m, __fmul2_rn(make_float2(omb1, omb1), g));
+  v = __ffma2_rn(b2, v, __fmul2_rn(__fmul2_rn(make_float2(omb2, omb2), g), g));
   const float2 vh = __fmul2_rn(v, make_float2(a.inv_bc2, a.inv_bc2));
   float2 root, inv;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root.x) : "f"(vh.x));
@@ -173,6 +180,29 @@ __device__ __forceinline__ void adamw_pair(const AdamScalars& a, float2 g, float
   const float2 upd = __fmul2_rn(__fmul2_rn(make_float2(a.step_size, a.step_size), m), inv);
   w = __ffma2_rn(make_float2(a.decay, a.decay), w, make_float2(-upd.x, -upd.y));
 }
+// The weights (1-beta1), (1-beta2) of the new gradient in the two moments, folded with the
+// clipping scale when the call clips by a norm known before the pass:
+//   s = min(1, max_norm / (sqrt(n2) + 1e-6));  m' = beta1 m + ((1-beta1) s) g;
+//   v' = beta2 v + ((1-beta2) s^2) g^2
+// -- AdamW on the clipped gradient s*g.  Without clipping the weights are the plain ones, bit
+// for bit.  Read after the dependency wait: n2 is what the previous call's last kernel wrote.
+struct GradWeights {
+  float omb1, omb2;
+};
+__device__ __forceinline__ GradWeights grad_weights(const AdamScalars& a, const double* clip_n2,
+                                                    double clip_max_norm) {
+  GradWeights w{a.omb1, a.omb2};
+  if (clip_n2) {
+    const double coef = clip_max_norm / (sqrt(__ldcg(clip_n2)) + 1e-6);
+    if (coef < 1.0) {
+      const float sc = static_cast<float>(coef);
+      w.omb1 *= sc;
+      w.omb2 *= sc * sc;
+    }
+  }
+  return w;
+}
+
 // max(x, +0) that keeps a NaN: the shifted one-pass variance can come out a few ulps below
 // zero and is clamped, but a NaN (a non-finite input, or squares that overflowed to inf - inf)
 // has to reach the sums so that the call reports ABS_FLAG_NONFINITE.  fmaxf would return 0.

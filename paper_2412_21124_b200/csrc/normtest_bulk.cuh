@@ -167,12 +167,14 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
   uint32_t tiles_done = 0;  // tiles this CTA has consumed so far: stage and phase bookkeeping
   bool waited = false;
   bool lost = false;        // a bounded wait ran out
+  GradWeights gw{prm.adam.omb1, prm.adam.omb2};
 
   for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
     const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, prm.grads, K, chunk);
     if (!waited) {  // everything above used kernel parameters only
       grid_dependency_wait();
       waited = true;
+      if (ADAM) gw = grad_weights(prm.adam, prm.clip_n2, prm.clip_max_norm);
     }
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
     CwMax cw;
@@ -181,7 +183,7 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
                       (prm.chunk_elems % kBulkTile == 0);
     if (!bulk) {
       cw.init(tid * GT::kVec);
-      chunk_rows_direct<GT, KB, EXACT, ADAM, STAT, NT>(prm, K, cg, acc_n2, acc_S, acc_Q, cw);
+      chunk_rows_direct<GT, KB, EXACT, ADAM, STAT, NT>(prm, K, cg, acc_n2, acc_S, acc_Q, cw, gw);
     } else {
       const int n_tiles = prm.chunk_elems / kBulkTile;
       const uint32_t tx_bytes = static_cast<uint32_t>(K * GB + (ADAM ? 3 * FB : 0));
@@ -254,7 +256,7 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
             cw.update(dev2.x, mean.x, li);
             cw.update(dev2.y, mean.y, li + 1);
           }
-          if (ADAM) adamw_pair(prm.adam, mean, w2[jp], m2[jp], v2[jp]);
+          if (ADAM) adamw_pair(prm.adam, gw.omb1, gw.omb2, mean, w2[jp], m2[jp], v2[jp]);
         }
         acc_n2 += static_cast<double>(row_n2);
         acc_S += static_cast<double>(row_S);

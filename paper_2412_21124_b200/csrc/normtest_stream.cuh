@@ -199,7 +199,7 @@ template <typename GT, int KB, bool EXACT, bool ADAM, int STAT, bool SPLIT = fal
 __device__ __noinline__ void scalar_row(const StreamParams& prm, const void* const* grads, int K,
                                         int64_t base, int64_t hi, int64_t chunk_lo,
                                         float* sums /* n2, S, Q of this thread-row */,
-                                        CwMax* cw) {
+                                        CwMax* cw, GradWeights gw) {
   constexpr int V = GT::kVec;
   constexpr bool WITHQ = STAT == kStatSumsQ;
   float row_n2 = 0.f, row_S = 0.f, row_Q = 0.f;
@@ -255,7 +255,7 @@ __device__ __noinline__ void scalar_row(const StreamParams& prm, const void* con
     if (prm.gbar) prm.gbar[i] = mean;
     if (ADAM) {
       float w = prm.p[i], m = prm.m[i], v = prm.v[i];
-      adamw_elem(prm.adam, mean, w, m, v);
+      adamw_elem(prm.adam, gw.omb1, gw.omb2, mean, w, m, v);
       prm.p[i] = w;
       prm.m[i] = m;
       prm.v[i] = v;
@@ -318,7 +318,8 @@ __device__ __forceinline__ ChunkGeometry chunk_geometry(const StreamParams& prm,
 template <typename GT, int KB, bool EXACT, bool ADAM, int STAT, int NT = kThreads>
 __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K,
                                                   const ChunkGeometry& cg, double& acc_n2,
-                                                  double& acc_S, double& acc_Q, CwMax& cw) {
+                                                  double& acc_S, double& acc_Q, CwMax& cw,
+                                                  GradWeights gw) {
   constexpr int V = GT::kVec;
   constexpr bool WITHQ = STAT == kStatSumsQ;
   constexpr bool CW = STAT == kStatCoordwise;
@@ -452,7 +453,7 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
               cw.update(dev2.x, mean.x, li);
               cw.update(dev2.y, mean.y, li + 1);
             }
-            if constexpr (ADAM) adamw_pair(prm.adam, mean, w2[jp], m2[jp], v2[jp]);
+            if constexpr (ADAM) adamw_pair(prm.adam, gw.omb1, gw.omb2, mean, w2[jp], m2[jp], v2[jp]);
           }
         } else {
 #pragma unroll
@@ -497,7 +498,7 @@ __device__ __forceinline__ void chunk_rows_direct(const StreamParams& prm, int K
       }
     } else if (base < hi) {
       float sums[3];
-      scalar_row<GT, KB, EXACT, ADAM, STAT>(prm, prm.grads, K, base, hi, cg.lo, sums, &cw);
+      scalar_row<GT, KB, EXACT, ADAM, STAT>(prm, prm.grads, K, base, hi, cg.lo, sums, &cw, gw);
       row_n2 = sums[0];
       row_S = sums[1];
       row_Q = sums[2];
@@ -555,16 +556,18 @@ __global__ void __launch_bounds__(kThreads, ((KB <= 8 && EXACT) ? 3 : ((KB <= 16
   __shared__ double red[kWarps * 3];
   const int K = EXACT ? KB : prm.K;
   bool waited = false;
+  GradWeights gw{prm.adam.omb1, prm.adam.omb2};
   for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
     const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, prm.grads, K, chunk);
     if (!waited) {  // everything above used kernel parameters only
       grid_dependency_wait();
       waited = true;
+      if (ADAM) gw = grad_weights(prm.adam, prm.clip_n2, prm.clip_max_norm);
     }
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
     CwMax cw;
     cw.init(static_cast<int>(threadIdx.x) * GT::kVec);
-    chunk_rows_direct<GT, KB, EXACT, ADAM, STAT>(prm, K, cg, acc_n2, acc_S, acc_Q, cw);
+    chunk_rows_direct<GT, KB, EXACT, ADAM, STAT>(prm, K, cg, acc_n2, acc_S, acc_Q, cw, gw);
     write_chunk_record<STAT>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, cw, red);
   }
 }
@@ -579,7 +582,8 @@ template <typename GT, int KB, bool EXACT, bool ADAM, int STAT>
 __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm,
                                                  const void* const* grads, int K,
                                                  const ChunkGeometry& cg, double& acc_n2,
-                                                 double& acc_S, double& acc_Q, CwMax& cw) {
+                                                 double& acc_S, double& acc_Q, CwMax& cw,
+                                                 GradWeights gw) {
   constexpr int V = GT::kVec;
   constexpr bool WITHQ = STAT == kStatSumsQ;
   constexpr bool CW = STAT == kStatCoordwise;
@@ -722,7 +726,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm,
           cw.update(tx, mean.x, li);
           cw.update(ty, mean.y, li + 1);
         }
-        if (ADAM) adamw_pair(prm.adam, mean, w2[pi], m2[pi], v2[pi]);
+        if (ADAM) adamw_pair(prm.adam, gw.omb1, gw.omb2, mean, w2[pi], m2[pi], v2[pi]);
       }
       if (prm.gbar) st_stream_16(prm.gbar + base, make_float4(gb[0], gb[1], gb[2], gb[3]));
       if (ADAM) {
@@ -733,7 +737,7 @@ __device__ __forceinline__ void chunk_rows_split(const StreamParams& prm,
       }
     } else if (base < hi) {
       float sums[3];
-      scalar_row<GT, KB, EXACT, ADAM, STAT, true>(prm, grads, K, base, hi, cg.lo, sums, &cw);
+      scalar_row<GT, KB, EXACT, ADAM, STAT, true>(prm, grads, K, base, hi, cg.lo, sums, &cw, gw);
       row_n2 = sums[0];
       row_S = sums[1];
       row_Q = sums[2];
@@ -750,16 +754,18 @@ __global__ void __launch_bounds__(kThreads, 2)
   __shared__ double red[kWarps * 3];
   const int K = EXACT ? KB : prm.K;
   bool waited = false;
+  GradWeights gw{prm.adam.omb1, prm.adam.omb2};
   for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
     const ChunkGeometry cg = chunk_geometry<GT, KB, EXACT, ADAM>(prm, prm.grads, K, chunk);
     if (!waited) {
       grid_dependency_wait();
       waited = true;
+      if (ADAM) gw = grad_weights(prm.adam, prm.clip_n2, prm.clip_max_norm);
     }
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
     CwMax cw;
     cw.init(static_cast<int>(threadIdx.x) * GT::kVec);
-    chunk_rows_split<GT, KB, EXACT, ADAM, STAT>(prm, prm.grads, K, cg, acc_n2, acc_S, acc_Q, cw);
+    chunk_rows_split<GT, KB, EXACT, ADAM, STAT>(prm, prm.grads, K, cg, acc_n2, acc_S, acc_Q, cw, gw);
     write_chunk_record<STAT>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, cw, red);
   }
 }
@@ -793,18 +799,20 @@ __global__ void __launch_bounds__(kThreads, 2)
   __shared__ double red[kWarps * 3];
   const int K = prm.K;
   bool waited = false;
+  GradWeights gw{prm.adam.omb1, prm.adam.omb2};
   for (int chunk = blockIdx.x; chunk < prm.n_chunks; chunk += gridDim.x) {
     const ChunkGeometry cg =
         chunk_geometry<GT, kInlineWorkers, false, ADAM>(prm, table.ptrs, K, chunk);
     if (!waited) {
       grid_dependency_wait();
       waited = true;
+      if (ADAM) gw = grad_weights(prm.adam, prm.clip_n2, prm.clip_max_norm);
     }
     double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
     CwMax cw;
     cw.init(static_cast<int>(threadIdx.x) * GT::kVec);
     chunk_rows_split<GT, kInlineWorkers, false, ADAM, STAT>(prm, table.ptrs, K, cg, acc_n2, acc_S,
-                                                            acc_Q, cw);
+                                                            acc_Q, cw, gw);
     write_chunk_record<STAT>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, cw, red);
   }
 }

@@ -297,6 +297,19 @@ def test_clipped_adamw_rejects(L):
     assert f(FAKE, FAKE, FAKE, FAKE, 10, r, 0, 1.0, FAKE, None) == binding.ABS_ERR_RANGE
 
 
+def test_clip_prev_rejects(L):
+    hp = _hp()
+    r = ctypes.byref(hp)
+    base = _nt_args(gbar=None)[:-1]
+    f = L.abs_normtest_adamw_clip_prev
+    far = [FAKE + 0x100000 * i for i in range(1, 4)]   # params, m, v apart from each other
+    assert f(*(base + far + [r, 1, 0.0, FAKE, None])) == binding.ABS_ERR_RANGE
+    assert f(*(base + far + [r, 1, math.nan, FAKE, None])) == binding.ABS_ERR_RANGE
+    assert f(*(base + far + [r, 1, 1.0, FAKE + 4, None])) == binding.ABS_ERR_ALIGN
+    assert f(*(base + [None] + far[1:] + [r, 1, 1.0, FAKE, None])) == binding.ABS_ERR_NULL
+    assert f(*(base + far + [r, 0, 1.0, None, None])) == binding.ABS_ERR_RANGE   # step, no clipping
+
+
 def test_mixed_precision_rejects(L):
     hp = binding.abs_adamw_hparams(1e-3, 0.9, 0.999, 1e-8, 0.1)
     r = ctypes.byref(hp)

@@ -551,6 +551,56 @@ def test_norm_test_then_clipped_adamw(max_norm, d, shift):
         assert torch.equal(q, views[0]) and torch.equal(mq, views[1]) and torch.equal(vq, views[2])
 
 
+@pytest.mark.parametrize("K,dtype,d", [(8, torch.bfloat16, 5 * 8192 + 777), (4, torch.float32, 50_001),
+                                       (12, torch.float32, 33_000), (32, torch.bfloat16, 20_481),
+                                       (100, torch.bfloat16, 9_999)],
+                         ids=["k8-bf16", "k4-f32", "k12-f32", "k32-bf16", "k100-bf16"])
+def test_fused_step_clipped_by_the_previous_norm(K, dtype, d):
+    """abs_normtest_adamw_clip_prev over three steps: step 1 unclipped (no previous norm), steps
+    2 and 3 clipped by the norm the step before wrote into the same stats buffer.  The oracle
+    clips by its own previous n2; the test's statistics stay those of the unclipped gradient."""
+    eta, b_cur, max_norm = 0.1, 64, 0.5
+    p, m, v = synth.adam_state(d, 1701, DEV, zero_moments=True)
+    ph, mh, vh = to_host(p), to_host(m), to_host(v)
+    stats = absnt.alloc_stats(d, 1, DEV)
+    gbar = torch.empty(d, dtype=torch.float32, device=DEV)
+    b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+    n2_prev, clipped_steps = None, 0
+    for step in (1, 2, 3):
+        grads, ref = make_case(K, d, dtype, eta, b_cur, seed=1700 + 10 * step + K)
+        absnt.abs_normtest_adamw_clip_prev(grads, eta, b_cur, stats, gbar, b_next, p, m, v, HP, step,
+                                           max_norm, stats if step > 1 else None)
+        torch.cuda.synchronize()
+        got = absnt.read_stats(stats)
+        assert_sum_close(got["n2"], ref["n2"], "n2")
+        assert_sum_close(got["S"], ref["S"], "S")
+        assert int(b_next.item()) == ref["b_next"]
+        assert_vec_close(gbar, ref["gbar"], "gbar")
+        hp = [f32(HP[k]) for k in ("lr", "beta1", "beta2", "eps", "weight_decay")]
+        if n2_prev is None:
+            w_ref, m_ref, v_ref = orc.adamw(ph, mh, vh, ref["gbar"], *hp, step)
+        else:
+            clipped_steps += orc.clip_scale(n2_prev, max_norm) < 1.0
+            w_ref, m_ref, v_ref = orc.adamw_clipped(ph, mh, vh, ref["gbar"], *hp, step, max_norm,
+                                                    n2_prev)
+        assert_vec_close(p, w_ref, "params")
+        assert_vec_close(m, m_ref, "m")
+        assert_vec_close(v, v_ref, "v")
+        # the next step starts from the library's stored state and the oracle's previous norm
+        ph, mh, vh = to_host(p), to_host(m), to_host(v)
+        n2_prev = ref["n2"]
+    assert clipped_steps == 2  # ||gbar|| is about 0.05 sqrt(d/K) + ..., well above 0.5
+    # a threshold the norm does not reach: the plain fused step, bit for bit
+    q, mq, vq = p.clone(), m.clone(), v.clone()
+    stats2 = absnt.alloc_stats(d, 1, DEV)
+    absnt.abs_normtest_adamw_clip_prev(grads, eta, b_cur, stats2, gbar, b_next, q, mq, vq, HP, 4,
+                                       1e9, stats)
+    absnt.abs_normtest_adamw(grads, eta, b_cur, stats, gbar, b_next, p, m, v, HP, 4)
+    torch.cuda.synchronize()
+    assert torch.equal(p, q) and torch.equal(m, mq) and torch.equal(v, vq)
+    assert torch.equal(stats[:2], stats2[:2])
+
+
 # ------------------------------------------------------------------- mixed precision
 def bf16_bits(t):
     return t.detach().cpu().view(torch.int16).numpy().view(np.uint16)
