@@ -304,10 +304,11 @@ int abs_normtest_adamw_noalloc(const void* const* grads, int K, int64_t d, abs_d
  *   stats_out  device, abs_persample_stats_bytes(b, d) bytes, 16-byte aligned; header
  *              as above with NORM = b-1 and one shard record; the diagnostic Q is not
  *              computed (NaN).  The buffer must be ZERO-FILLED before its first use with
- *              this call (for a given b, d): the thread blocks of its last kernel count
- *              themselves off in a ticket counter kept in this buffer; the counter is back
- *              at zero when the call completes, so the buffer can be reused as it is.  Zero it again after a call that returned ABS_ERR_CUDA, or
- *              before using it with another (b, d).
+ *              this call: the thread blocks of its last kernel count themselves off in a
+ *              ticket counter kept in this buffer (the doubles right after the shard record,
+ *              at the same place for every b and d); the counter is back at zero when the call
+ *              completes, so the buffer can be reused as it is, for any shape it is large
+ *              enough for.  Zero it again after a call that returned ABS_ERR_CUDA.
  *   gbar_out   device, d floats;  b_next_out device, one int64
  */
 int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs_dtype dtype,

@@ -423,10 +423,10 @@ size_t abs_persample_stats_bytes(int64_t b, int64_t d) {
   const int rpb = persample_rows_per_block(b, d);
   const size_t nrb = static_cast<size_t>((b + rpb - 1) / rpb);
   const size_t nmb = static_cast<size_t>((d + kPsThreads - 1) / kPsThreads);
-  // header, one shard record, {n2, S} per CTA of the merge pass, {sum, M2} per (row block,
-  // column), and the ticket counter (one double's worth)
-  return sizeof(double) * (ABS_STATS_HEADER + ABS_SHARD_STRIDE + 2 * nmb +
-                           2 * nrb * static_cast<size_t>(d) + 1);
+  // header, one shard record, the ticket counter (two doubles' worth, at a fixed place),
+  // {n2, S} per CTA of the merge pass, {sum, M2} per (row block, column)
+  return sizeof(double) * (ABS_STATS_HEADER + ABS_SHARD_STRIDE + kPsTicketDoubles + 2 * nmb +
+                           2 * nrb * static_cast<size_t>(d));
 }
 
 int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
@@ -595,10 +595,12 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
   prm.n_row_blocks = static_cast<int>(nrb);
   const int64_t nmb = (d + kPsThreads - 1) / kPsThreads;  // CTAs of the merge pass
   if (nmb > INT32_MAX) return ABS_ERR_RANGE;
-  prm.cb_rec = stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE;
+  // the ticket counter sits at the same place whatever b and d are, so a buffer that has
+  // served one shape (and therefore holds zero there) serves any other shape it is large enough for
+  prm.tickets = reinterpret_cast<unsigned int*>(stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE);
+  prm.cb_rec = stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE + kPsTicketDoubles;
   prm.ws_sum = prm.cb_rec + 2 * nmb;
   prm.ws_m2 = prm.ws_sum + nrb * d;
-  prm.tickets = reinterpret_cast<unsigned int*>(prm.ws_m2 + nrb * d);
   prm.gbar = gbar_out;
   prm.stats = stats;
   prm.b_next = b_next_out;

@@ -266,6 +266,7 @@ __global__ void __launch_bounds__(kPsThreads, kPsCtasPerSM)
 }
 
 // Pass 2 and the decision (see the top of the file).
+constexpr int kPsTicketDoubles = 2;    // room for the ticket counter in stats_out (keeps 16-byte alignment)
 constexpr int kPsMergeInFlight = 16;  // row blocks of a column in flight at once
 
 __global__ void __launch_bounds__(kPsThreads)

@@ -801,6 +801,15 @@ def test_persample_stats_buffer_is_reusable_and_calls_are_bit_identical():
         torch.cuda.synchronize()
         assert torch.equal(stats[:12].view(torch.int64), outs[0][0].view(torch.int64))
         assert torch.equal(gbar, outs[0][1])
+    # the same buffer, now full of another shape's records, serves a smaller problem as it is
+    G2 = G[:300, :1234].contiguous()
+    gbar2 = torch.empty(1234, dtype=torch.float32, device=DEV)
+    absnt.abs_persample_norm_test(G2, 0.1, stats, gbar2, b_next)
+    torch.cuda.synchronize()
+    ref2 = orc.persample(G2.cpu().numpy(), 0.1)
+    assert_sum_close(float(stats[1]), ref2["S"], "S")
+    assert_sum_close(float(stats[0]), ref2["n2"], "n2")
+    assert_vec_close(gbar2, ref2["gbar"], "gbar")
 
 
 def test_persample_more_rows_than_one_grid_dimension_of_512_row_blocks():
