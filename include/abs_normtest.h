@@ -405,6 +405,18 @@ int abs_schedule_test_due(const abs_schedule* s);
 /* Returns ABS_OK, ABS_ERR_NULL, or ABS_ERR_RANGE (b_test < 1; the state is then unchanged). */
 int abs_schedule_advance(abs_schedule* s, int64_t b_test);
 
+/*
+ * Self-test of the bounded waits (no counterpart in the paper).  The staged kernels wait for
+ * their asynchronous copies on shared-memory barriers, and every such wait gives up after a
+ * fixed number of polls (2^18, about one second on a B200) instead of spinning for ever; a kernel whose wait gave up
+ * poisons its partial sums, so the call reports ABS_FLAG_NONFINITE.  This entry point runs
+ * that wait on a barrier nothing will complete, for `polls` polls (1 .. 2^18), and writes
+ * out[0] = 1 if the wait gave up (it must), out[1] = the time it took in nanoseconds
+ * (device, two int64).  It shows that the give-up path ends by itself and how long the full
+ * limit lasts on the device at hand.
+ */
+int abs_selftest_bounded_wait(int polls, int64_t* out, abs_stream_t stream);
+
 const char* abs_status_string(int status);
 
 /* The cudaError_t of the most recent ABS_ERR_CUDA on this thread (0 if none). */

@@ -102,6 +102,8 @@ def lib():
     L.abs_schedule_test_due.argtypes = [ptr]
     L.abs_schedule_advance.restype = cint
     L.abs_schedule_advance.argtypes = [ptr, i64]
+    L.abs_selftest_bounded_wait.restype = cint
+    L.abs_selftest_bounded_wait.argtypes = [cint, ptr, ptr]
     L.abs_status_string.restype = ctypes.c_char_p
     L.abs_status_string.argtypes = [cint]
     L.abs_last_cuda_error.restype = cint
@@ -500,6 +502,17 @@ def abs_combine_sums(rows, norm, eta, b_cur):
 def abs_noalloc_fits(d, shard_offsets=None):
     offs, n_shards = _offsets(shard_offsets)
     return bool(lib().abs_noalloc_fits(int(d), offs, n_shards))
+
+
+def abs_selftest_bounded_wait(polls, stream=None):
+    """Runs the staged kernels' bounded wait on a barrier nothing completes.  Returns
+    (gave_up, nanoseconds)."""
+    out = torch.zeros(2, dtype=torch.int64, device="cuda")
+    rc = lib().abs_selftest_bounded_wait(int(polls), out.data_ptr(), _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_selftest_bounded_wait")
+    gave_up, ns = out.tolist()  # synchronises
+    return bool(gave_up), int(ns)
 
 
 def abs_round_batch(b_next, J, M):

@@ -223,6 +223,25 @@ int make_layout(int64_t d, const int64_t* shard_offsets, int n_shards, bool fuse
   return ABS_OK;
 }
 
+// A wait of the staged kernels' kind on a barrier that nothing will ever complete: one thread
+// polls `polls` times with the same instruction as mbar_wait_bounded and reports that it gave
+// up and how long that took.  Nothing here can hang: the loop has a fixed trip count.
+__global__ void bounded_wait_selftest_kernel(int polls, long long* out) {
+  __shared__ uint64_t bar;
+  grid_dependency_wait();
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    long long t0, t1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    bool completed = false;
+    for (int i = 0; i < polls && !completed; ++i) completed = mbar_try_wait(&bar, 0u);
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+    out[0] = completed ? 0 : 1;
+    out[1] = t1 - t0;
+  }
+}
+
 // ---------------------------------------------------------------------------------------
 // abs_normtest_adamw_noalloc: the fused step with its chunk records in an array that is
 // part of the library image, for callers that cannot allocate device memory.
@@ -668,6 +687,16 @@ int64_t abs_round_batch(int64_t b_next, int64_t J, int64_t M) {
   const int64_t jm = J * M;
   const int64_t micro = (b_next + jm - 1) / jm;
   return J * (M * micro);
+}
+
+int abs_selftest_bounded_wait(int polls, int64_t* out, abs_stream_t stream) {
+  if (!out) return ABS_ERR_NULL;
+  if (polls < 1 || polls > kBulkWaitLimit) return ABS_ERR_RANGE;
+  if (misaligned(out, 8)) return ABS_ERR_ALIGN;
+  const cudaError_t e = launch_pdl(bounded_wait_selftest_kernel, dim3(1), dim3(32),
+                                   static_cast<cudaStream_t>(stream), polls,
+                                   reinterpret_cast<long long*>(out));
+  return e == cudaSuccess ? ABS_OK : cuda_fail(e);
 }
 
 const char* abs_status_string(int status) {

@@ -24,7 +24,10 @@
 
 namespace absnt {
 
-constexpr int kBulkWaitLimit = 1 << 22;  // mbarrier polls before giving up
+// mbarrier polls before giving up.  A poll that fails returns after the hardware's own
+// suspend time, measured at 3.95 us on a B200, so the limit is about one second: four orders
+// of magnitude above any wait a landing copy needs, short enough to end a lost one soon.
+constexpr int kBulkWaitLimit = 1 << 18;
 constexpr int kSmemPerSM = 224 * 1024;   // budget for dynamic shared memory per SM
 
 // bytes of one stage of `tile` coordinates

@@ -224,6 +224,22 @@ def test_edge_cases_at_the_large_chunk_size():
         _check_vectors_where_finite(gbar, ref, state, 3, {d - 2})
 
 
+def test_a_wait_that_nothing_completes_gives_up_by_itself():
+    """The staged kernels wait for their asynchronous copies with a bounded number of polls.
+    Here that wait runs on a barrier nothing will ever complete: it must give up, and the time
+    per poll says how long the full limit of 2^18 polls lasts (printed; about a second)."""
+    for polls in (1, 64, 4096):
+        gave_up, ns = absnt.abs_selftest_bounded_wait(polls)
+        assert gave_up and ns > 0
+    per_poll = ns / 4096.0
+    print("bounded wait: %.1f ns per poll, 2^18 polls = %.2f s" % (per_poll, per_poll * 2 ** 18 / 1e9))
+    assert per_poll * 2 ** 18 < 10e9   # the full limit ends within seconds
+    with pytest.raises(absnt.AbsError):
+        absnt.abs_selftest_bounded_wait(0)
+    with pytest.raises(absnt.AbsError):
+        absnt.abs_selftest_bounded_wait(2 ** 18 + 1)
+
+
 # ------------------------------------------------------------------- per-sample kernels
 def _persample(G, eta):
     b, d = G.shape
