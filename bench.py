@@ -223,6 +223,7 @@ def run_ours(args, d):
     ev[1].record(stream)
     torch.cuda.synchronize()
     est_ms = max(ev[0].elapsed_time(ev[1]), 1e-3)          # a first, untimed block
+    est_ms = adist.max_over_ranks(est_ms, dev)             # every rank must time the same blocks
     n_blocks = int(min(MAX_BLOCKS, max(MIN_BLOCKS, -(-TIMED_REGION_MS // est_ms))))
     events = [torch.cuda.Event(enable_timing=True) for _ in range(n_blocks + 1)]
     adist.barrier(dev)
