@@ -60,7 +60,9 @@ def _jobs():
 
 def _compile(job, nvcc, verbose):
     obj, src, defines = job
-    cmd = [nvcc] + NVCC_FLAGS + defines + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", obj, src]
+    extra = os.environ.get("ABS_NVCC_EXTRA", "").split()  # e.g. -D switches for A/B builds
+    cmd = ([nvcc] + NVCC_FLAGS + defines + extra + (["-Xptxas", "-v"] if verbose else [])
+           + ["-c", "-o", obj, src])
     out = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
     if out.returncode != 0:
         raise RuntimeError("nvcc failed on %s %s:\n%s" % (os.path.basename(src), " ".join(defines),
