@@ -34,7 +34,9 @@ namespace absnt {
 // What a kernel accumulates besides gbar: the two sums of the test always; the diagnostic
 // Q = sum_k ||g_k||^2 on request; or, for the coordinate-wise test (Sec. 4, Proposition 1),
 // the largest per-coordinate ratio sum_k (g_k[i]-gbar_i)^2 / gbar_i^2 and where it occurs.
-enum StatMode { kStatSums = 0, kStatSumsQ = 1, kStatCoordwise = 2 };
+// kStatNone: no statistics at all (the stand-alone AdamW update runs as the one-worker fused
+// kernel in this mode: nothing is reduced, no chunk record is written).
+enum StatMode { kStatSums = 0, kStatSumsQ = 1, kStatCoordwise = 2, kStatNone = 3 };
 
 // Running maximum of the per-coordinate ratio within one thread, then one chunk.  The ratio is
 // formed in fp32 with the hardware reciprocal (2^-22 relative).  A coordinate with zero
@@ -516,6 +518,7 @@ template <int STAT, int NT = kThreads>
 __device__ __forceinline__ void write_chunk_record(const StreamParams& prm, int chunk,
                                                    int64_t chunk_lo, double acc_n2, double acc_S,
                                                    double acc_Q, CwMax cw, double* red) {
+  if constexpr (STAT == kStatNone) return;
   constexpr bool WITHQ = STAT == kStatSumsQ;
   constexpr bool CW = STAT == kStatCoordwise;
   __shared__ float cw_r[NT / 32];

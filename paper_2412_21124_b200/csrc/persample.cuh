@@ -381,7 +381,8 @@ __global__ void __launch_bounds__(kPsThreads)
   }
 }
 
-// Stand-alone AdamW (Algorithm 1, AdamW lines), in place.  With `n2_dev` non-null the
+// Stand-alone AdamW (Algorithm 1, AdamW lines), in place, for vectors below 2^25 coordinates
+// (larger ones run as the one-worker fused kernel).  With `n2_dev` non-null the
 // gradient is first clipped by global norm: g <- g * min(1, max_norm / (sqrt(n2) + 1e-6)),
 // n2 = ||gbar||^2 read from the stats header a preceding norm test wrote on the device
 // (no host round trip).  Clipping is what the paper's experiments add to Algorithm 1.
@@ -392,11 +393,8 @@ __global__ void __launch_bounds__(kThreads)
                  const double* __restrict__ n2_dev, double max_norm, uint16_t* __restrict__ p16) {
   const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
   grid_dependency_wait();
-  float scale = 1.f;
-  if (n2_dev) {
-    const double coef = max_norm / (sqrt(*n2_dev) + 1e-6);
-    scale = coef < 1.0 ? static_cast<float>(coef) : 1.f;
-  }
+  // the clipping scale is folded into the weights of the new gradient (see GradWeights)
+  const GradWeights gw = grad_weights(a, n2_dev, max_norm);
   if (VEC) {
     const int64_t nvec = d >> 2;
     int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
@@ -407,18 +405,18 @@ __global__ void __launch_bounds__(kThreads)
       const float4 g1 = __ldcs(reinterpret_cast<const float4*>(g) + j);
       float4 p0 = ld_state_16(p + 4 * i), m0 = ld_state_16(m + 4 * i), v0 = ld_state_16(v + 4 * i);
       float4 p1 = ld_state_16(p + 4 * j), m1 = ld_state_16(m + 4 * j), v1 = ld_state_16(v + 4 * j);
-      adamw_elem(a, a.omb1, a.omb2, scale * g0.x, p0.x, m0.x, v0.x);
-      adamw_elem(a, a.omb1, a.omb2, scale * g0.y, p0.y, m0.y, v0.y);
-      adamw_elem(a, a.omb1, a.omb2, scale * g0.z, p0.z, m0.z, v0.z);
-      adamw_elem(a, a.omb1, a.omb2, scale * g0.w, p0.w, m0.w, v0.w);
+      adamw_elem(a, gw.omb1, gw.omb2, g0.x, p0.x, m0.x, v0.x);
+      adamw_elem(a, gw.omb1, gw.omb2, g0.y, p0.y, m0.y, v0.y);
+      adamw_elem(a, gw.omb1, gw.omb2, g0.z, p0.z, m0.z, v0.z);
+      adamw_elem(a, gw.omb1, gw.omb2, g0.w, p0.w, m0.w, v0.w);
       st_stream_16(p + 4 * i, p0);
       st_stream_16(m + 4 * i, m0);
       st_stream_16(v + 4 * i, v0);
       if (p16) st_bf16x4(p16 + 4 * i, p0);
-      adamw_elem(a, a.omb1, a.omb2, scale * g1.x, p1.x, m1.x, v1.x);
-      adamw_elem(a, a.omb1, a.omb2, scale * g1.y, p1.y, m1.y, v1.y);
-      adamw_elem(a, a.omb1, a.omb2, scale * g1.z, p1.z, m1.z, v1.z);
-      adamw_elem(a, a.omb1, a.omb2, scale * g1.w, p1.w, m1.w, v1.w);
+      adamw_elem(a, gw.omb1, gw.omb2, g1.x, p1.x, m1.x, v1.x);
+      adamw_elem(a, gw.omb1, gw.omb2, g1.y, p1.y, m1.y, v1.y);
+      adamw_elem(a, gw.omb1, gw.omb2, g1.z, p1.z, m1.z, v1.z);
+      adamw_elem(a, gw.omb1, gw.omb2, g1.w, p1.w, m1.w, v1.w);
       st_stream_16(p + 4 * j, p1);
       st_stream_16(m + 4 * j, m1);
       st_stream_16(v + 4 * j, v1);
@@ -427,10 +425,10 @@ __global__ void __launch_bounds__(kThreads)
     if (i < nvec) {
       const float4 gg = __ldcs(reinterpret_cast<const float4*>(g) + i);
       float4 pp = ld_state_16(p + 4 * i), mm = ld_state_16(m + 4 * i), vv = ld_state_16(v + 4 * i);
-      adamw_elem(a, a.omb1, a.omb2, scale * gg.x, pp.x, mm.x, vv.x);
-      adamw_elem(a, a.omb1, a.omb2, scale * gg.y, pp.y, mm.y, vv.y);
-      adamw_elem(a, a.omb1, a.omb2, scale * gg.z, pp.z, mm.z, vv.z);
-      adamw_elem(a, a.omb1, a.omb2, scale * gg.w, pp.w, mm.w, vv.w);
+      adamw_elem(a, gw.omb1, gw.omb2, gg.x, pp.x, mm.x, vv.x);
+      adamw_elem(a, gw.omb1, gw.omb2, gg.y, pp.y, mm.y, vv.y);
+      adamw_elem(a, gw.omb1, gw.omb2, gg.z, pp.z, mm.z, vv.z);
+      adamw_elem(a, gw.omb1, gw.omb2, gg.w, pp.w, mm.w, vv.w);
       st_stream_16(p + 4 * i, pp);
       st_stream_16(m + 4 * i, mm);
       st_stream_16(v + 4 * i, vv);
@@ -440,7 +438,7 @@ __global__ void __launch_bounds__(kThreads)
     const int64_t t = (nvec << 2) + threadIdx.x;
     if (blockIdx.x == 0 && t < d) {
       float pp = p[t], mm = m[t], vv = v[t];
-      adamw_elem(a, a.omb1, a.omb2, scale * g[t], pp, mm, vv);
+      adamw_elem(a, gw.omb1, gw.omb2, g[t], pp, mm, vv);
       p[t] = pp;
       m[t] = mm;
       v[t] = vv;
@@ -450,7 +448,7 @@ __global__ void __launch_bounds__(kThreads)
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < d;
          i += stride) {
       float pp = p[i], mm = m[i], vv = v[i];
-      adamw_elem(a, a.omb1, a.omb2, scale * g[i], pp, mm, vv);
+      adamw_elem(a, gw.omb1, gw.omb2, g[i], pp, mm, vv);
       p[i] = pp;
       m[i] = mm;
       v[i] = vv;

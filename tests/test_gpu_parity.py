@@ -514,6 +514,47 @@ def test_adamw_step_sequence(d, shift):
         check_guards(b, d, shift)
 
 
+@pytest.mark.parametrize("shift", [0, 1])
+def test_adamw_step_large_vector(shift):
+    """From 2^25 coordinates on the update runs as the one-worker fused kernel (bulk-staged, with
+    its element-wise path for a misaligned vector): plain, clipped and with the bf16 copy, against
+    the oracle; and the clipped update agrees bit for bit with the small-vector kernel's on the
+    same values."""
+    d = (1 << 25) + 4097
+    g = shifted_copy(synth.worker_grads([d], 1, torch.float32, 1290, DEV)[0], shift)
+    p, m, v = (shifted_copy(t, shift) for t in synth.adam_state(d, 1291, DEV, zero_moments=False))
+    p0, m0, v0 = to_host(p), to_host(m), to_host(v)
+    g64 = to_host(g).astype(np.float64)
+    absnt.abs_adamw_step(p, g, m, v, HP, 7)
+    torch.cuda.synchronize()
+    w_ref, m_ref, v_ref = oracle_adamw(orc, p0, m0, v0, g64, HP, 7)
+    assert_vec_close(p, w_ref, "params")
+    assert_vec_close(m, m_ref, "m")
+    assert_vec_close(v, v_ref, "v")
+    # clipped, with the bf16 copy; n2 comes from a stats header as a norm test would write it
+    n2 = float((g.double() ** 2).sum())
+    stats = torch.zeros(absnt.binding.ABS_STATS_HEADER, dtype=torch.float64, device=DEV)
+    stats[absnt.binding.ABS_STAT_N2] = n2
+    p16 = torch.zeros(d, dtype=torch.bfloat16, device=DEV)
+    p1, m1, v1 = to_host(p), to_host(m), to_host(v)
+    absnt.abs_adamw_step_mixed(p, g, m, v, p16, HP, 8, max_norm=1.0, stats_in=stats)
+    torch.cuda.synchronize()
+    assert orc.clip_scale(n2, 1.0) < 1.0
+    w_ref, m_ref, v_ref = orc.adamw_clipped(p1, m1, v1, g64, f32(HP["lr"]), f32(HP["beta1"]),
+                                            f32(HP["beta2"]), f32(HP["eps"]),
+                                            f32(HP["weight_decay"]), 8, 1.0, n2)
+    assert_vec_close(p, w_ref, "params")
+    assert_vec_close(m, m_ref, "m")
+    assert_vec_close(v, v_ref, "v")
+    assert np.array_equal(bf16_bits(p16), orc.bf16_round(to_host(p)))
+    # the first 100,000 coordinates through the small-vector kernel: identical bits
+    n = 100_000
+    q, mq, vq = (torch.from_numpy(x[:n].copy()).to(DEV) for x in (p1, m1, v1))
+    absnt.abs_adamw_step_clipped(q, g[:n].clone(), mq, vq, HP, 8, 1.0, stats)
+    torch.cuda.synchronize()
+    assert torch.equal(q, p[:n]) and torch.equal(mq, m[:n]) and torch.equal(vq, v[:n])
+
+
 @pytest.mark.parametrize("max_norm", [1.0, 0.05, 1e3])
 @pytest.mark.parametrize("d,shift", [(100_003, 0), (50_001, 1)])
 def test_norm_test_then_clipped_adamw(max_norm, d, shift):
