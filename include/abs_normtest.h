@@ -115,7 +115,12 @@ size_t abs_persample_stats_bytes(int64_t b, int64_t d);
  * the shard records added in shard order.
  *
  *   grads          host array of K device pointers, each d elements of `dtype`,
- *                  aligned to the element size (16-byte alignment is faster, not required)
+ *                  aligned to the element size (16-byte alignment is faster, not required).
+ *                  They are only read, with plain loads and non-multicast bulk copies, so a
+ *                  buffer may also live on another GPU whose memory the current device can
+ *                  address (peer access enabled, or an opened inter-process handle): the
+ *                  gradient exchange of Sec. 3.2 is then the kernel's own loads.  Every
+ *                  output must be memory of the current device.
  *   K              1..ABS_MAX_WORKERS (1024 = 4 workers x 256 accumulation steps, the largest
  *                  layout of the paper's Table 5, should the J*M micro-batch gradients of a
  *                  step serve as the samples of the estimator)

@@ -160,6 +160,18 @@ def _check_one_device(*tensors):
                              % (cur, t.device))
 
 
+def _check_peer_grads(grads):
+    """Gradient buffers that may live on other GPUs: each on the current device or on one whose
+    memory the current device can address (peer access; a buffer opened from another process's
+    handle counts as living on its owner's device)."""
+    cur = torch.cuda.current_device()
+    for g in grads:
+        if not g.is_cuda:
+            raise ValueError("gradient buffers must be CUDA tensors, got %s" % g.device)
+        if g.device.index != cur and not torch.cuda.can_device_access_peer(cur, g.device.index):
+            raise ValueError("cuda:%d cannot address the memory of %s" % (cur, g.device))
+
+
 def _stream(stream):
     if stream is None:
         return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
@@ -279,7 +291,11 @@ def abs_adamw_step_clipped(params, gbar, m, v, hparams, step, max_norm, stats_in
 
 
 def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, params, m, v, hparams,
-                       step, shard_offsets=None, stream=None, _entry="abs_normtest_adamw"):
+                       step, shard_offsets=None, stream=None, _entry="abs_normtest_adamw",
+                       peer_grads=False):
+    """The fused step.  `peer_grads=True` lets the gradient buffers (read-only inputs) live on
+    other GPUs whose memory the current device can address: the kernel then loads them over
+    NVLink (plain loads and non-multicast bulk copies); everything written stays local."""
     table, K, d, code = _grad_table(grads)
     offs, n_shards = _offsets(shard_offsets)
     for t, name in ((params, "params"), (m, "m"), (v, "v")):
@@ -288,7 +304,11 @@ def abs_normtest_adamw(grads, eta, b_cur, stats_out, gbar_out, b_next_out, param
         _check_f32_vec(gbar_out, d, "gbar_out")
     _check_stats(stats_out, abs_stats_bytes(d, n_shards))
     _check_b_next(b_next_out)
-    _check_one_device(*grads, stats_out, gbar_out, b_next_out, params, m, v)
+    if peer_grads:
+        _check_peer_grads(grads)
+        _check_one_device(stats_out, gbar_out, b_next_out, params, m, v)
+    else:
+        _check_one_device(*grads, stats_out, gbar_out, b_next_out, params, m, v)
     hp = _hparams(hparams)
     rc = getattr(lib(), _entry)(table, K, d, code, offs, n_shards, float(eta), int(b_cur),
                                 stats_out.data_ptr(),

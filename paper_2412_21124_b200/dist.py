@@ -13,9 +13,16 @@ cross the wire.  This module holds that small host-side logic:
                       the fused step on this rank's index range followed by that exchange:
                       the multi-GPU form of FSDP-Norm (Sec. 3.3; Algorithm 1 with the shard
                       sums "concatenated")
+  share_across_ranks, ddp_normtest_adamw
+                      the DDP layout of Sec. 3.2 (DDP-Norm): every rank holds the gradient of
+                      its own minibatch for the whole vector and makes it addressable by its
+                      peers; rank r then runs the fused call on index range r of all ranks'
+                      buffers, so the gradient exchange is the kernel's own loads over NVLink
+                      (no all-reduce of d elements, no second all-reduce for the variance)
   max_over_ranks      max-reduction used for timing
 """
 import os
+import pickle
 
 import torch
 import torch.distributed as dist
@@ -41,12 +48,16 @@ def init_from_env(backend=None):
     return rank, world, local_rank
 
 
-def rank_range(d, rank, world):
-    """[lo, hi) of the flat vector owned by `rank`: equal contiguous ranges, the first
-    d % world ranks holding one extra coordinate."""
-    q, r = divmod(int(d), int(world))
+def rank_range(d, rank, world, align=1):
+    """[lo, hi) of the flat vector owned by `rank`: equal contiguous ranges of whole units of
+    `align` coordinates (the last unit may be short), the first ranks holding one extra unit
+    where the units do not divide evenly.  align = 1: the first d % world ranks hold one
+    extra coordinate."""
+    units = -(-int(d) // int(align))
+    q, r = divmod(units, int(world))
     lo = rank * q + min(rank, r)
-    return lo, lo + q + (1 if rank < r else 0)
+    hi = lo + q + (1 if rank < r else 0)
+    return min(lo * align, int(d)), min(hi * align, int(d))
 
 
 def combine_rank_sums(n2, S, Q, K, eta, b_cur, device="cpu", group=None):
@@ -93,6 +104,82 @@ def sharded_normtest_adamw(grads_local, eta, b_cur, stats_out, gbar_out, b_next_
                                params_local, m_local, v_local, hparams, step)
     local = stats_out.view(torch.float64)[binding.ABS_STAT_N2:binding.ABS_STAT_Q + 1]
     return binding.abs_combine_sums(_gather_rank_rows(local, group), len(grads_local), eta, b_cur)
+
+
+def share_across_ranks(t, group=None):
+    """Makes this rank's CUDA tensor `t` addressable by every rank of the group and returns the
+    list, in rank order, of all ranks' tensors as this process sees them (its own entry is `t`
+    itself; the others are views of the owners' device memory, opened from inter-process
+    handles, living on the owner's device index).  Collective; call it once per buffer and
+    keep `t` alive while any rank uses the views.  Every process must see all GPUs of the node
+    under the same indices."""
+    from multiprocessing.reduction import ForkingPickler
+    import torch.multiprocessing.reductions  # noqa: F401  (registers the CUDA tensor reducer)
+    if not (dist.is_initialized() and dist.get_world_size(group) > 1):
+        return [t]
+    if not t.is_cuda:
+        raise ValueError("only CUDA tensors can be shared across ranks")
+    world, rank = dist.get_world_size(group), dist.get_rank(group)
+    blobs = [None] * world
+    dist.all_gather_object(blobs, bytes(ForkingPickler.dumps(t)), group=group)
+    return [t if r == rank else pickle.loads(blobs[r]) for r in range(world)]
+
+
+def _all_ranks_reached(group=None):
+    """Everything this rank has enqueued on its current stream so far is complete, on every
+    rank, before anything enqueued after this call runs.  NCCL: a one-element all-reduce on
+    the stream (the host does not wait); other backends: stream synchronise + host barrier."""
+    if not (dist.is_initialized() and dist.get_world_size(group) > 1):
+        return
+    if dist.get_backend(group) == "nccl":
+        dist.all_reduce(torch.zeros(1, device="cuda"), group=group)
+    else:
+        torch.cuda.current_stream().synchronize()
+        dist.barrier(group=group)
+
+
+kDdpRangeAlign = 64   # coordinates: rank ranges start on 128-byte (bf16) / 256-byte (fp32) lines
+
+
+def ddp_normtest_adamw(peer_grads, eta, b_cur, stats_out, b_next_out, params, m_local, v_local,
+                       hparams, step, group=None):
+    """DDP-Norm step (Sec. 3.2; Algorithm 1 with J workers) with one process per GPU.
+
+    `peer_grads` is `share_across_ranks` of the ranks' own gradient buffers (rank j's entry
+    holds the gradient of worker j's minibatch for the whole flat vector, d elements).  Rank r
+    runs the fused norm-test + AdamW call on index range r (`rank_range` with
+    align = kDdpRangeAlign, so that every range starts on a vector boundary) of ALL J buffers:
+    its loads of the other ranks' ranges cross NVLink once, which is the reduce-scatter of
+    the gradient average done by the kernel's own loads, and the variance sum of Eq. 5 comes
+    out of the same pass.  `params` is this rank's full replica (d fp32 values) and is
+    updated in place on range r; `m_local`, `v_local` are the moments of range r only (no
+    other rank needs them).  Then the three sums per rank are gathered and added in rank
+    order (every rank takes the same decision from the same bits) and the updated ranges are
+    broadcast so that every replica of `params` is whole again.
+
+    Ordering: the call starts with a rendezvous -- no rank reads a peer's gradient before that
+    peer's stream has finished writing it -- and the closing broadcasts are the second one:
+    when they return on a rank, every rank's kernel has read what it needed, so the gradient
+    buffers may be overwritten.  Returns the dict of `abs_combine_sums`."""
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    rank = dist.get_rank(group) if dist.is_initialized() else 0
+    if len(peer_grads) != world:
+        raise ValueError("peer_grads must hold one buffer per rank")
+    d = params.numel()
+    lo, hi = rank_range(d, rank, world, kDdpRangeAlign)
+    _all_ranks_reached(group)
+    binding.abs_normtest_adamw([g[lo:hi] for g in peer_grads], eta, b_cur, stats_out, None,
+                               b_next_out, params[lo:hi], m_local, v_local, hparams, step,
+                               peer_grads=True)
+    local = stats_out.view(torch.float64)[binding.ABS_STAT_N2:binding.ABS_STAT_Q + 1]
+    out = binding.abs_combine_sums(_gather_rank_rows(local, group), world, eta, b_cur)
+    if world > 1:
+        for r in range(world):
+            r_lo, r_hi = rank_range(d, r, world, kDdpRangeAlign)
+            if r_hi > r_lo:
+                dist.broadcast(params[r_lo:r_hi], src=dist.get_global_rank(group, r)
+                               if group is not None else r, group=group)
+    return out
 
 
 def barrier(device=None):

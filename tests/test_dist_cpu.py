@@ -56,6 +56,17 @@ def test_rank_ranges_cover():
             assert lo == prev and hi >= lo
             prev = hi
         assert prev == d
+    # whole units of `align` coordinates: every range starts on a unit boundary, the ranges still
+    # tile [0, d), and ranks beyond the last unit get empty ranges
+    for d, w, al in ((1000, 3, 64), (64, 4, 64), (65, 4, 64), (124_439_808, 8, 64), (7, 2, 64)):
+        prev = 0
+        for r in range(w):
+            lo, hi = adist.rank_range(d, r, w, al)
+            assert lo == prev and hi >= lo and (lo % al == 0 or lo == d)
+            prev = hi
+        assert prev == d
+        sizes = [adist.rank_range(d, r, w, al) for r in range(w)]
+        assert max(h - l for l, h in sizes) - min(h - l for l, h in sizes) < 2 * al
 
 
 def test_two_rank_combine_matches_oracle():
