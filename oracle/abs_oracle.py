@@ -201,6 +201,32 @@ def round_batch(b_next, J, M):
     return int(lib().abs_oracle_round_batch(int(b_next), int(J), int(M)))
 
 
+def _least(holds, lo, hi):
+    """Smallest integer in [lo, hi] at which the monotone predicate `holds` (false, ..., false,
+    true, ..., true) is true; it must be true at hi.  Bisection, so that any size is exact."""
+    assert holds(hi)
+    while lo < hi:
+        mid = (lo + hi) // 2
+        if holds(mid):
+            hi = mid
+        else:
+            lo = mid + 1
+    return lo
+
+
+def _greatest(holds, lo, hi):
+    """Largest integer in [lo, hi] at which the monotone predicate `holds` (true, ..., true,
+    false, ..., false) is true; it must be true at lo."""
+    assert holds(lo)
+    while lo < hi:
+        mid = (lo + hi + 1) // 2
+        if holds(mid):
+            lo = mid
+        else:
+            hi = mid - 1
+    return lo
+
+
 class Schedule:
     """Algorithm 1's loop state around the test, in Python integers (exact at any size): the
     If branch (microbatch rounded up, minibatch = M * microbatch, global = J * minibatch), the
@@ -222,20 +248,26 @@ class Schedule:
         return self.b < self.b_max and self.step % self.interval == 0
 
     def advance(self, b_test):
-        used = self.b
+        """One pass of the loop body after the test.  The new layout is stated as what it has
+        to satisfy and found by search over the integers (`_least`, `_greatest`), not by a
+        rounding formula."""
+        J, used = self.J, self.b
         target = min(b_test, self.b_max)
-        if target > self.b:
+        if target > self.b:   # the If branch (the Else branch changes nothing)
+            def covers(M, micro):
+                return J * M * micro >= target
+            # the paper's M, unless even the largest allowed microbatch does not cover the
+            # target with it: then the smallest count of accumulation steps that does
             M = self.M
-            micro = -(-target // (self.J * M))
-            if self.max_micro and micro > self.max_micro:
-                M = -(-target // (self.J * self.max_micro))
-                micro = -(-target // (self.J * M))
-            b = self.J * M * micro
-            if b > self.b_max:
-                micro = self.b_max // (self.J * M)
-                b = self.J * M * micro
-            if micro >= 1 and b > self.b:
-                self.M, self.micro, self.b = M, micro, b
+            if self.max_micro and not covers(M, self.max_micro):
+                M = _least(lambda c: covers(c, self.max_micro), self.M, target)
+            # the smallest microbatch that covers the target ...
+            micro = _least(lambda u: covers(M, u), 1, target)
+            if J * M * micro > self.b_max:
+                # ... or, should that pass the cap, the largest one that stays under it
+                micro = _greatest(lambda u: J * M * u <= self.b_max, 0, micro)
+            if micro >= 1 and J * M * micro > self.b:   # only ever an increase
+                self.M, self.micro, self.b = M, micro, J * M * micro
         self.samples += used
         self.step += 1
 
