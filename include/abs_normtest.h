@@ -141,6 +141,35 @@ int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                   const int64_t* shard_offsets, int n_shards, double eta, int64_t b_cur,
                   void* stats_out, float* gbar_out, int64_t* b_next_out, abs_stream_t stream);
 
+/*
+ * The norm test over gradients that arrive a few at a time (gradient accumulation: Sec. 3.2,
+ * "the technique of gradient accumulation is applied"; Algorithm 1's accumulation loop), in
+ * O(d) memory: the K new buffers are merged into the running mean of the count_in gradients
+ * that the earlier calls of this step merged, and into the running variance sum.
+ *
+ *   count_in = 0     starts a step: `mean_inout` and the sums in `stats_inout` are only written.
+ *   count_in > 0     `mean_inout` holds the mean of the count_in gradients so far and
+ *                    `stats_inout` is the buffer the previous call of the step wrote (its shard
+ *                    records carry the sums; the same d and shard table must be passed).
+ * After the call `mean_inout` is the mean of all count_in + K gradients (after the last call of
+ * the step: gbar of Algorithm 1), and the header, the shard records and b_next_out are those of
+ * the test over all of them, with 1/(count_in + K) in place of 1/J in Eq. 5 -- what
+ * abs_norm_test returns when given all the buffers at once, up to rounding: the running mean is
+ * rounded to fp32 once per call (relative 2^-24 each, so gbar agrees with the one-call result
+ * to about 2^-24 sqrt(calls) of its magnitude), the sums agree to the usual 1e-6.  Per call
+ * K*s + 8 bytes per coordinate cross HBM (the new gradients once, the mean read and written).
+ * The caller advances count_in by K between calls.  K is 1..64 here; Q is not computed.
+ *
+ *   mean_inout     device, d floats, aligned to 4 bytes; must not overlap a gradient buffer
+ *   stats_inout    device, abs_stats_bytes(d, n_shards) bytes, 16-byte aligned
+ *   other arguments as for abs_norm_test
+ * Non-finite values, once merged, stay in the mean and the sums until a call with count_in = 0.
+ */
+int abs_norm_test_accumulate(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                             const int64_t* shard_offsets, int n_shards, int64_t count_in,
+                             double eta, int64_t b_cur, void* stats_inout, float* mean_inout,
+                             int64_t* b_next_out, abs_stream_t stream);
+
 /* abs_norm_test that also accumulates the diagnostic Q = sum_k sum_i g_k[i]^2, per shard and
  * in total (the identity S = Q - K*n2 checks a run's sums against each other). */
 int abs_norm_test_q(const void* const* grads, int K, int64_t d, abs_dtype dtype,

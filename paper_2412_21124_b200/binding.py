@@ -79,6 +79,9 @@ def lib():
     L.abs_norm_test_coordwise.argtypes = list(L.abs_norm_test.argtypes)
     L.abs_norm_test_q.restype = cint
     L.abs_norm_test_q.argtypes = list(L.abs_norm_test.argtypes)
+    L.abs_norm_test_accumulate.restype = cint
+    L.abs_norm_test_accumulate.argtypes = [ptr, cint, i64, cint, ptr, cint, i64, dbl, i64, ptr,
+                                           ptr, ptr, ptr]
     L.abs_normtest_adamw_coordwise.restype = cint
     L.abs_normtest_adamw_coordwise.argtypes = list(L.abs_normtest_adamw.argtypes)
     L.abs_normtest_adamw_mixed.restype = cint
@@ -246,6 +249,26 @@ def abs_norm_test(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offs
                                 _stream(stream))
     if rc != ABS_OK:
         raise AbsError(rc, _entry)
+
+
+def abs_norm_test_accumulate(grads, count_in, eta, b_cur, stats_inout, mean_inout, b_next_out,
+                             shard_offsets=None, stream=None):
+    """Merges the K new gradient buffers into the running mean (`mean_inout`, d floats) and the
+    running sums (`stats_inout`) of the `count_in` gradients merged by the earlier calls of this
+    step; count_in = 0 starts a step.  After the call the outputs are those of the test over all
+    count_in + K gradients."""
+    table, K, d, code = _grad_table(grads)
+    offs, n_shards = _offsets(shard_offsets)
+    _check_f32_vec(mean_inout, d, "mean_inout")
+    _check_stats(stats_inout, abs_stats_bytes(d, n_shards))
+    _check_b_next(b_next_out)
+    _check_one_device(*grads, stats_inout, mean_inout, b_next_out)
+    rc = lib().abs_norm_test_accumulate(table, K, d, code, offs, n_shards, int(count_in),
+                                        float(eta), int(b_cur), stats_inout.data_ptr(),
+                                        mean_inout.data_ptr(), b_next_out.data_ptr(),
+                                        _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_norm_test_accumulate")
 
 
 def abs_norm_test_q(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offsets=None,

@@ -1,0 +1,245 @@
+// Carry-in form of the norm test: the worker (or micro-batch) gradients of one step arrive a
+// few at a time -- as they do under gradient accumulation -- and are merged into a running
+// state of O(d) memory instead of being kept side by side.
+//
+// State between the calls of a step: the running mean of the n gradients merged so far (d fp32
+// values: the gradient-accumulation buffer itself, holding the mean instead of the sum) and, per
+// shard, the running sum of squared deviations about that mean (in the shard records of the
+// stats buffer).  Merging m new gradients g_1..g_m into (n, mean, M2), per coordinate, with the
+// old mean as the centre c (for n = 0: c = g_1):
+//     sd = sum_k (g_k - c)        q = sum_k (g_k - c)^2
+//     mean' = c + sd / (n + m)    M2' = M2 + q - sd^2 / (n + m)
+// which is the pooled-variance update (law of total variance) written about the old mean: the
+// term taken off q is never larger than q (Cauchy-Schwarz) and small against it once n >> m,
+// so nothing cancels.  After the last call mean' is gbar of Algorithm 1 ("Compute the batch
+// gradient"), sum_i M2'_i the variance sum of Eq. 5, and n2 = sum_i mean'_i^2 is recomputed by
+// every call (each call visits every coordinate).  Deviations and their squares are fp32 per
+// coordinate, accumulated per group of workers and then over groups (as in the many-worker
+// kernel), fp64 from the thread-row upwards.
+//
+// The chunk records have the layout of the other streaming kernels and go through the same
+// finalize kernel; the carry enters as one more addend: the CTA of a shard's first chunk adds
+// the shard's previous sum to its own partial.  Few workers per call leave little in flight,
+// so for m <= 4 a thread loads several thread-rows before it consumes the first.
+#pragma once
+#include "normtest_stream.cuh"
+
+namespace absnt {
+
+struct AccumCarry {
+  double n_prev;            // gradients merged by the earlier calls of this step; 0 starts a step
+  float inv_total;          // 1 / (n_prev + K)
+  const double* shard_rec;  // shard records left by the previous call (slot 1: its sum S_s)
+};
+
+// Accumulators of one thread-row (four coordinates as two packed pairs).
+template <typename GT>
+struct AccumRow {
+  static constexpr int P = 2;
+  float2 c[P], neg_c[P];  // the centre
+  float2 s2[P], g2[P];    // squared deviations: closed groups, the open group
+  float2 sd[P], gd[P];    // deviations: the same
+  // the centre: the running mean, or (first call of a step) the first gradient, set by the caller
+  __device__ __forceinline__ void init(const float4& centre) {
+#pragma unroll
+    for (int pi = 0; pi < P; ++pi) s2[pi] = g2[pi] = sd[pi] = gd[pi] = make_float2(0.f, 0.f);
+    c[0] = make_float2(centre.x, centre.y);
+    c[1] = make_float2(centre.z, centre.w);
+#pragma unroll
+    for (int pi = 0; pi < P; ++pi) neg_c[pi] = make_float2(-c[pi].x, -c[pi].y);
+  }
+  __device__ __forceinline__ void init_from(const typename GT::raw_t& first_gradient) {
+    const float2 a = GT::pair(first_gradient, 0), b = GT::pair(first_gradient, 1);
+    init(make_float4(a.x, a.y, b.x, b.y));
+  }
+  __device__ __forceinline__ void add(const typename GT::raw_t& raw) {
+#pragma unroll
+    for (int pi = 0; pi < P; ++pi) {
+      const float2 dv = __fadd2_rn(GT::pair(raw, pi), neg_c[pi]);
+      gd[pi] = __fadd2_rn(gd[pi], dv);
+      g2[pi] = __ffma2_rn(dv, dv, g2[pi]);
+    }
+  }
+  __device__ __forceinline__ void close_group() {
+#pragma unroll
+    for (int pi = 0; pi < P; ++pi) {
+      s2[pi] = __fadd2_rn(s2[pi], g2[pi]);
+      sd[pi] = __fadd2_rn(sd[pi], gd[pi]);
+      g2[pi] = gd[pi] = make_float2(0.f, 0.f);
+    }
+  }
+  // the new means of the four coordinates; adds their squares and the M2 increments
+  __device__ __forceinline__ float4 finish(float inv_total, float& row_n2, float& row_S) {
+    float mean[4];
+#pragma unroll
+    for (int pi = 0; pi < P; ++pi) {
+      const float2 it = make_float2(inv_total, inv_total);
+      const float2 dm = __fmul2_rn(sd[pi], it);
+      const float2 mu = __fadd2_rn(c[pi], dm);
+      const float2 t = __ffma2_rn(make_float2(-sd[pi].x, -sd[pi].y), dm, s2[pi]);
+      mean[2 * pi] = mu.x;
+      mean[2 * pi + 1] = mu.y;
+      row_n2 = fmaf(mu.x, mu.x, row_n2);
+      row_n2 = fmaf(mu.y, mu.y, row_n2);
+      row_S += clamp_nonneg(t.x);
+      row_S += clamp_nonneg(t.y);
+    }
+    return make_float4(mean[0], mean[1], mean[2], mean[3]);
+  }
+};
+
+// One thread-row with element-wise, bounds-checked accesses (ragged end of a shard, streams
+// that are not 16-byte aligned): the operations of AccumRow in the same order.
+template <typename GT>
+__device__ __noinline__ void accumulate_scalar_row(const StreamParams& prm, const AccumCarry& cy,
+                                                   int K, int64_t base, int64_t hi, float* sums) {
+  constexpr int H = split_group<GT, false>();
+  const bool carry = cy.n_prev > 0.0;
+  float row_n2 = 0.f, row_S = 0.f;
+  for (int e = 0; e < GT::kVec; ++e) {
+    const int64_t i = base + e;
+    if (i >= hi) break;
+    const float c = carry ? prm.gbar[i] : GT::load1(prm.grads[0], i);
+    float s2 = 0.f, g2 = 0.f, sd = 0.f, gd = 0.f;
+    for (int k = 0; k < K; ++k) {
+      const float dv = GT::load1(prm.grads[k], i) - c;
+      gd += dv;
+      g2 = fmaf(dv, dv, g2);
+      if ((k + 1) % H == 0 || k + 1 == K) {
+        s2 += g2;
+        sd += gd;
+        g2 = gd = 0.f;
+      }
+    }
+    const float dm = sd * cy.inv_total;
+    const float mu = c + dm;
+    row_n2 = fmaf(mu, mu, row_n2);
+    row_S += clamp_nonneg(fmaf(-sd, dm, s2));
+    prm.gbar[i] = mu;
+  }
+  sums[0] = row_n2;
+  sums[1] = row_S;
+}
+
+// ROWS > 1: calls with at most KR workers load ROWS thread-rows (ROWS * K gradient vectors and the
+// ROWS mean vectors: 128 bytes of gradients per thread for ROWS * KR = 8 vectors of 16 bytes or
+// 16 of 8 bytes) before the first is consumed; rows are consumed in order, so the sums have the
+// shape of the ROWS = 1 kernel and both give the same bits.
+template <typename GT, int ROWS, int KR>
+__global__ void __launch_bounds__(kThreads, 3)
+    normtest_accumulate_kernel(const __grid_constant__ StreamParams prm,
+                               const __grid_constant__ AccumCarry cy) {
+  static_assert(GT::kVec == 4, "four coordinates per thread-row");
+  constexpr int V = 4;
+  constexpr int H = split_group<GT, false>();
+  __shared__ double red[kWarps * 3];
+  const int K = prm.K;
+  const int tid = threadIdx.x;
+  const int chunk = blockIdx.x;
+  const bool carry = cy.n_prev > 0.0;
+  const ChunkGeometry cg = chunk_geometry<GT, kInlineWorkers, false, false>(prm, prm.grads, K, chunk);
+  // does this chunk open its shard?  (the shard: the last s with chunk_prefix[s] <= chunk)
+  int lo_s = 0, hi_s = prm.n_shards;
+  while (hi_s - lo_s > 1) {
+    const int mid = (lo_s + hi_s) >> 1;
+    if (prm.chunk_prefix[mid] <= chunk) lo_s = mid; else hi_s = mid;
+  }
+  const bool opens_shard = chunk == prm.chunk_prefix[lo_s];
+  grid_dependency_wait();
+
+  double acc_n2 = 0.0, acc_S = 0.0, acc_Q = 0.0;
+  const int64_t hi = cg.hi;
+  int64_t row_lo = cg.lo;
+  auto vec_ptr = [&](int k, int64_t base) {
+    return reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) + base;
+  };
+
+  if constexpr (ROWS > 1) {
+    while (cg.aligned && row_lo + static_cast<int64_t>(ROWS) * kThreads * V <= hi) {
+      typename GT::raw_t raw[ROWS][KR];
+      float4 mo[ROWS];
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r) {
+        const int64_t base = row_lo + (static_cast<int64_t>(r) * kThreads + tid) * V;
+#pragma unroll
+        for (int k = 0; k < KR; ++k)
+          if (k < K) raw[r][k] = GT::load_vec(vec_ptr(k, base));
+        mo[r] = carry ? ld_state_16(prm.gbar + base) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r) {
+        const int64_t base = row_lo + (static_cast<int64_t>(r) * kThreads + tid) * V;
+        AccumRow<GT> acc;
+        if (carry) acc.init(mo[r]); else acc.init_from(raw[r][0]);
+#pragma unroll
+        for (int k = 0; k < KR; ++k)
+          if (k < K) acc.add(raw[r][k]);
+        acc.close_group();
+        float row_n2 = 0.f, row_S = 0.f;
+        st_stream_16(prm.gbar + base, acc.finish(cy.inv_total, row_n2, row_S));
+        acc_n2 += static_cast<double>(row_n2);
+        acc_S += static_cast<double>(row_S);
+      }
+      row_lo += static_cast<int64_t>(ROWS) * kThreads * V;
+    }
+  }
+
+  for (; row_lo < hi; row_lo += kThreads * V) {
+    const int64_t base = row_lo + static_cast<int64_t>(tid) * V;
+    float row_n2 = 0.f, row_S = 0.f;
+    if (cg.aligned && row_lo + kThreads * V <= hi) {
+      AccumRow<GT> acc;
+      bool need_centre = !carry;  // uniform across the CTA
+      if (carry) acc.init(ld_state_16(prm.gbar + base));
+      // N consecutive workers from k0: all loads first, then the arithmetic
+      auto piece = [&](int k0, auto n_tag) {
+        constexpr int N = decltype(n_tag)::value;
+        typename GT::raw_t raw[N];
+#pragma unroll
+        for (int k = 0; k < N; ++k) raw[k] = GT::load_vec(vec_ptr(k0 + k, base));
+        if (need_centre) {
+          acc.init_from(raw[0]);
+          need_centre = false;
+        }
+#pragma unroll
+        for (int k = 0; k < N; ++k) acc.add(raw[k]);
+      };
+      int k0 = 0;
+#pragma unroll 1
+      for (; k0 + H <= K; k0 += H) {
+        piece(k0, std::integral_constant<int, H>{});
+        acc.close_group();
+      }
+      if (H > 8 && ((K - k0) & 8)) {
+        piece(k0, std::integral_constant<int, 8>{});
+        k0 += 8;
+      }
+      if ((K - k0) & 4) {
+        piece(k0, std::integral_constant<int, 4>{});
+        k0 += 4;
+      }
+      if ((K - k0) & 2) {
+        piece(k0, std::integral_constant<int, 2>{});
+        k0 += 2;
+      }
+      if ((K - k0) & 1) piece(k0, std::integral_constant<int, 1>{});
+      acc.close_group();  // adds exact zeros when K is a multiple of H
+      st_stream_16(prm.gbar + base, acc.finish(cy.inv_total, row_n2, row_S));
+    } else if (base < hi) {
+      float sums[2];
+      accumulate_scalar_row<GT>(prm, cy, K, base, hi, sums);
+      row_n2 = sums[0];
+      row_S = sums[1];
+    }
+    acc_n2 += static_cast<double>(row_n2);
+    acc_S += static_cast<double>(row_S);
+  }
+  // the shard's sum so far rides on the first thread's partial of the shard's first chunk
+  if (carry && opens_shard && tid == 0)
+    acc_S += __ldcg(cy.shard_rec + static_cast<int64_t>(lo_s) * ABS_SHARD_STRIDE + 1);
+  CwMax unused;
+  unused.init(0);
+  write_chunk_record<kStatSums>(prm, chunk, cg.lo, acc_n2, acc_S, acc_Q, unused, red);
+}
+
+}  // namespace absnt

@@ -48,6 +48,8 @@ def bytes_per_call(call, d, K, esz, gbar, b):
         return (K * esz + 4) * d
     if call == "adamw":
         return 28 * d
+    if call == "accumulate":  # the K new gradients once, the running mean read and written
+        return (K * esz + 8) * d
     return esz * b * d
 
 
@@ -65,14 +67,14 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
     sets = []
     for i in range(n_sets):
         s = {}
-        if call in ("fused", "normtest"):
+        if call in ("fused", "normtest", "accumulate"):
             sizes = _sizes(d)
             sig = synth.per_tensor_sigma(sizes, 11)
             s["grads"] = synth.worker_grads(sizes, K, tdt, 100 + i, dev, sigma=sig)
             s["stats"] = B.alloc_stats(d, n_shards, dev)
         if call in ("fused", "adamw"):
             s["p"], s["m"], s["v"] = synth.adam_state(d, 200 + i, dev, zero_moments=False)
-        if call in ("normtest", "adamw") or gbar:
+        if call in ("normtest", "adamw", "accumulate") or gbar:
             s["gbar"] = torch.zeros(d, dtype=torch.float32, device=dev)
             if call == "adamw":
                 s["gbar"].normal_().mul_(0.02)
@@ -101,6 +103,9 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
             B.abs_adamw_step_mixed(s["p"], s["gbar"], s["m"], s["v"], s["p16"], HP, 100 + i)
         elif call == "adamw":
             B.abs_adamw_step(s["p"], s["gbar"], s["m"], s["v"], HP, 100 + i)
+        elif call == "accumulate":  # a later call of a step: the running mean is read and written
+            B.abs_norm_test_accumulate(s["grads"], 8 * K, 0.1, 512, s["stats"], s["gbar"],
+                                       s["b_next"], shard_offsets=offs)
         else:
             B.abs_persample_norm_test(s["G"], 0.1, s["stats"], s["gbar"], s["b_next"])
 
@@ -193,6 +198,8 @@ REPORT_POINTS = (
        ("fused", GPT2, 8, "bf16", 1, {"coordwise": True}),
        ("fused", GPT2, 4, "f32", 1, {"coordwise": True}),
        ("fused", GPT2, 32, "bf16", 1, {"coordwise": True})]
+    # the carry-in form: K new gradients merged into the running mean per call
+    + [("accumulate", GPT2, K, dt, 1, {}) for K in (1, 2, 4, 8, 16) for dt in ("bf16", "f32")]
     # the paper's own model sizes (Table 4), J = 4 workers, bf16
     + [("fused", d, 4, "bf16", 1, {}) for d in (304_600_000, 1_100_000_000, 3_400_000_000)])
 
@@ -275,7 +282,7 @@ def format_markdown(path):
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("--call", choices=["fused", "normtest", "adamw", "persample"], default="fused")
+    ap.add_argument("--call", choices=["fused", "normtest", "adamw", "persample", "accumulate"], default="fused")
     ap.add_argument("--d", type=int, default=33_554_432)
     ap.add_argument("--K", type=int, default=8)
     ap.add_argument("--dtype", choices=["bf16", "f32"], default="bf16")

@@ -263,6 +263,42 @@ def test_norm_test_rejects(L, over, status):
     assert L.abs_norm_test(*_nt_args(**over)) == status
 
 
+def _acc_args(**over):
+    K = over.pop("K", 2)
+    table = over.pop("table", (ctypes.c_void_p * 64)(*([FAKE] * 64)))
+    a = dict(grads=table, K=K, d=100, dtype=0, offs=None, n_shards=1, count_in=0, eta=0.1,
+             b_cur=8, stats=FAKE, mean=FAKE, b_next=FAKE, stream=None)
+    a.update(over)
+    return [a[k] for k in ("grads", "K", "d", "dtype", "offs", "n_shards", "count_in", "eta",
+                           "b_cur", "stats", "mean", "b_next", "stream")]
+
+
+@pytest.mark.parametrize("over,status", [
+    (dict(grads=None), binding.ABS_ERR_NULL),
+    (dict(stats=None), binding.ABS_ERR_NULL),
+    (dict(mean=None), binding.ABS_ERR_NULL),
+    (dict(b_next=None), binding.ABS_ERR_NULL),
+    (dict(dtype=2), binding.ABS_ERR_DTYPE),
+    (dict(K=0), binding.ABS_ERR_RANGE),
+    (dict(K=65), binding.ABS_ERR_RANGE),          # more per call than the carry-in form takes
+    (dict(count_in=-1), binding.ABS_ERR_RANGE),
+    (dict(d=0), binding.ABS_ERR_RANGE),
+    (dict(b_cur=0), binding.ABS_ERR_RANGE),
+    (dict(eta=0.0), binding.ABS_ERR_RANGE),
+    (dict(eta=math.nan), binding.ABS_ERR_RANGE),
+    (dict(stats=FAKE + 8), binding.ABS_ERR_ALIGN),
+    (dict(mean=FAKE + 2), binding.ABS_ERR_ALIGN),
+    (dict(table=(ctypes.c_void_p * 32)(FAKE, 0)), binding.ABS_ERR_NULL),
+    (dict(offs=_offs(0, 99), n_shards=1), binding.ABS_ERR_SHARDS),
+    # the running mean is read and written while the gradients are read: no overlap allowed
+    (dict(), binding.ABS_ERR_ALIAS),
+    (dict(table=(ctypes.c_void_p * 32)(FAKE + 0x100000, FAKE + 0x200000), mean=FAKE + 0x100000 + 40,
+          stats=FAKE + 0x300000, b_next=FAKE + 0x400000), binding.ABS_ERR_ALIAS),
+])
+def test_accumulate_rejects(L, over, status):
+    assert L.abs_norm_test_accumulate(*_acc_args(**over)) == status
+
+
 def _hp(**over):
     v = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
     v.update(over)
