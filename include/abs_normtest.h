@@ -142,8 +142,8 @@ int abs_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
                   void* stats_out, float* gbar_out, int64_t* b_next_out, abs_stream_t stream);
 
 /*
- * The norm test over gradients that arrive a few at a time (gradient accumulation: Sec. 3.2,
- * "the technique of gradient accumulation is applied"; Algorithm 1's accumulation loop), in
+ * The norm test over gradients that arrive a few at a time (gradient accumulation: Sec. 3.2
+ * names it for minibatches that exceed a worker's memory; Algorithm 1's accumulation loop), in
  * O(d) memory: the K new buffers are merged into the running mean of the count_in gradients
  * that the earlier calls of this step merged, and into the running variance sum.
  *
