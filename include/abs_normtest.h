@@ -170,6 +170,29 @@ int abs_norm_test_accumulate(const void* const* grads, int K, int64_t d, abs_dty
                              double eta, int64_t b_cur, void* stats_inout, float* mean_inout,
                              int64_t* b_next_out, abs_stream_t stream);
 
+/*
+ * The closing call of a step in the carry-in form, fused with AdamW (Algorithm 1: the test,
+ * then the AdamW lines on the batch gradient): merges the last K buffers as
+ * abs_norm_test_accumulate does and applies the update with the final mean in the same pass,
+ * so the mean is consumed in registers: K*s + 4 + 24 bytes per coordinate instead of
+ * K*s + 8 for the merge plus 28 for abs_adamw_step.
+ *
+ *   mean_in        device, d floats: the running mean of the count_in gradients merged so far
+ *                  (read only; NULL allowed when count_in = 0, which makes this call the whole
+ *                  step, as abs_normtest_adamw is)
+ *   gbar_out       device, d floats, or NULL when the final mean is not wanted; may be
+ *                  `mean_in` itself (updated in place), must not overlap it otherwise
+ *   params, m, v, hparams, step   as for abs_normtest_adamw
+ * ABS_ERR_CUDA after the first launch: as for abs_normtest_adamw (the update may be enqueued).
+ */
+int abs_norm_test_accumulate_adamw(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                                   const int64_t* shard_offsets, int n_shards, int64_t count_in,
+                                   double eta, int64_t b_cur, void* stats_inout,
+                                   const float* mean_in, float* gbar_out, int64_t* b_next_out,
+                                   float* params, float* m, float* v,
+                                   const abs_adamw_hparams* hparams, int64_t step,
+                                   abs_stream_t stream);
+
 /* abs_norm_test that also accumulates the diagnostic Q = sum_k sum_i g_k[i]^2, per shard and
  * in total (the identity S = Q - K*n2 checks a run's sums against each other). */
 int abs_norm_test_q(const void* const* grads, int K, int64_t d, abs_dtype dtype,

@@ -82,6 +82,9 @@ def lib():
     L.abs_norm_test_accumulate.restype = cint
     L.abs_norm_test_accumulate.argtypes = [ptr, cint, i64, cint, ptr, cint, i64, dbl, i64, ptr,
                                            ptr, ptr, ptr]
+    L.abs_norm_test_accumulate_adamw.restype = cint
+    L.abs_norm_test_accumulate_adamw.argtypes = [ptr, cint, i64, cint, ptr, cint, i64, dbl, i64,
+                                                 ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i64, ptr]
     L.abs_normtest_adamw_coordwise.restype = cint
     L.abs_normtest_adamw_coordwise.argtypes = list(L.abs_normtest_adamw.argtypes)
     L.abs_normtest_adamw_mixed.restype = cint
@@ -269,6 +272,35 @@ def abs_norm_test_accumulate(grads, count_in, eta, b_cur, stats_inout, mean_inou
                                         _stream(stream))
     if rc != ABS_OK:
         raise AbsError(rc, "abs_norm_test_accumulate")
+
+
+def abs_norm_test_accumulate_adamw(grads, count_in, eta, b_cur, stats_inout, mean_in, gbar_out,
+                                   b_next_out, params, m, v, hparams, step, shard_offsets=None,
+                                   stream=None):
+    """The closing call of a step in the carry-in form, fused with AdamW: merges the last K
+    buffers into the running mean `mean_in` (None when count_in = 0) and updates params / m / v
+    with the final mean in the same pass; `gbar_out` (None, or `mean_in` itself) receives it."""
+    table, K, d, code = _grad_table(grads)
+    offs, n_shards = _offsets(shard_offsets)
+    for t, name in ((params, "params"), (m, "m"), (v, "v")):
+        _check_f32_vec(t, d, name)
+    for t, name in ((mean_in, "mean_in"), (gbar_out, "gbar_out")):
+        if t is not None:
+            _check_f32_vec(t, d, name)
+    if count_in > 0 and mean_in is None:
+        raise ValueError("count_in > 0 needs the running mean")
+    _check_stats(stats_inout, abs_stats_bytes(d, n_shards))
+    _check_b_next(b_next_out)
+    _check_one_device(*grads, stats_inout, mean_in, gbar_out, b_next_out, params, m, v)
+    hp = _hparams(hparams)
+    rc = lib().abs_norm_test_accumulate_adamw(
+        table, K, d, code, offs, n_shards, int(count_in), float(eta), int(b_cur),
+        stats_inout.data_ptr(), mean_in.data_ptr() if mean_in is not None else None,
+        gbar_out.data_ptr() if gbar_out is not None else None, b_next_out.data_ptr(),
+        params.data_ptr(), m.data_ptr(), v.data_ptr(), ctypes.byref(hp), int(step),
+        _stream(stream))
+    if rc != ABS_OK:
+        raise AbsError(rc, "abs_norm_test_accumulate_adamw")
 
 
 def abs_norm_test_q(grads, eta, b_cur, stats_out, gbar_out, b_next_out, shard_offsets=None,

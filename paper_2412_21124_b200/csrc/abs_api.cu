@@ -399,6 +399,118 @@ int run_norm_test(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   return ABS_OK;
 }
 
+// The one body behind abs_norm_test_accumulate and its closing form with AdamW.
+int run_accumulate(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                   const int64_t* shard_offsets, int n_shards, int64_t count_in, double eta,
+                   int64_t b_cur, void* stats_inout, const float* mean_in, float* gbar_out,
+                   int64_t* b_next_out, float* params, float* m, float* v,
+                   const abs_adamw_hparams* hparams, int64_t step, bool fused,
+                   abs_stream_t stream) {
+  if (!grads || !stats_inout || !b_next_out) return ABS_ERR_NULL;
+  if (count_in > 0 && !mean_in) return ABS_ERR_NULL;
+  if (!fused && !gbar_out) return ABS_ERR_NULL;
+  if (fused && (!params || !m || !v)) return ABS_ERR_NULL;
+  if (dtype != ABS_F32 && dtype != ABS_BF16) return ABS_ERR_DTYPE;
+  if (K < 1 || K > kInlineWorkers || d < 1 || b_cur < 1) return ABS_ERR_RANGE;
+  if (count_in < 0 || count_in > (int64_t{1} << 40)) return ABS_ERR_RANGE;
+  if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
+  if (fused) {
+    const int rch = check_hparams(hparams, step);
+    if (rch != ABS_OK) return rch;
+  }
+  const size_t esz = (dtype == ABS_F32) ? 4 : 2;
+  for (int k = 0; k < K; ++k) {
+    if (!grads[k]) return ABS_ERR_NULL;
+    if (misaligned(grads[k], esz)) return ABS_ERR_ALIGN;
+  }
+  if (count_in == 0) mean_in = nullptr;  // not read
+  if (misaligned(stats_inout, 16) || misaligned(b_next_out, 8) || misaligned(mean_in, 4) ||
+      misaligned(gbar_out, 4))
+    return ABS_ERR_ALIGN;
+  if (fused && (misaligned(params, 4) || misaligned(m, 4) || misaligned(v, 4))) return ABS_ERR_ALIGN;
+  Layout L;
+  const int rc = make_layout(d, shard_offsets, n_shards, false, &L);
+  if (rc != ABS_OK) return rc;
+  const size_t ud = static_cast<size_t>(d);
+  const Range outs[] = {{gbar_out, ud * 4}, {params, ud * 4}, {m, ud * 4}, {v, ud * 4},
+                        {stats_inout, abs_stats_bytes(d, L.n_shards)}, {b_next_out, 8}};
+  if (any_alias(grads, K, ud * esz, outs, 6)) return ABS_ERR_ALIAS;
+  // the running mean may be updated in place (mean_in == gbar_out: every coordinate is read and
+  // written by the same thread) but must not overlap anything else that is written
+  if (mean_in)
+    for (const Range& o : outs) {
+      const bool in_place = o.p == gbar_out && gbar_out == mean_in;
+      if (o.p && !in_place && overlaps(o.p, o.bytes, mean_in, ud * 4)) return ABS_ERR_ALIAS;
+    }
+  const int finalize_ctas = finalize_max_cluster();
+
+  double* stats = static_cast<double*>(stats_inout);
+  StreamParams prm;
+  std::memset(&prm, 0, sizeof prm);
+  for (int k = 0; k < K; ++k) prm.grads[k] = grads[k];
+  std::memcpy(prm.shard_off, L.shard_off, sizeof(int64_t) * (L.n_shards + 1));
+  std::memcpy(prm.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
+  prm.d = d;
+  prm.K = K;
+  prm.n_shards = L.n_shards;
+  prm.n_chunks = L.n_chunks;
+  prm.chunk_elems = L.chunk_elems;
+  prm.gbar = gbar_out;
+  prm.p = params;
+  prm.m = m;
+  prm.v = v;
+  prm.chunk_out = stats + ABS_STATS_HEADER + static_cast<size_t>(L.n_shards) * ABS_SHARD_STRIDE;
+  if (fused) prm.adam = make_adam(hparams, step);
+  const double total = static_cast<double>(count_in) + static_cast<double>(K);
+  AccumCarry cy;
+  cy.n_prev = static_cast<double>(count_in);
+  cy.inv_total = static_cast<float>(1.0 / total);
+  cy.mean_in = mean_in;
+  cy.shard_rec = stats + ABS_STATS_HEADER;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const dim3 grid(static_cast<unsigned>(L.n_chunks)), block(kThreads);
+  cudaError_t e;
+  // few gradients per call: several thread-rows in flight per thread, 128 bytes of gradients
+  // either way (fp32: 16-byte vectors, bf16: 8-byte vectors; eight rows for one or two bf16
+  // gradients spill, four rows serve them).  With AdamW the state vectors are in flight as
+  // well: two rows up to four gradients, one beyond.
+  if (fused) {
+    if (dtype == ABS_F32)
+      e = K <= 4 ? launch_pdl(normtest_accumulate_kernel<F32, 2, 4, true>, grid, block, st, prm, cy)
+                 : launch_pdl(normtest_accumulate_kernel<F32, 1, 1, true>, grid, block, st, prm, cy);
+    else
+      e = K <= 4   ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 4, true>, grid, block, st, prm, cy)
+          : K <= 8 ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 8, true>, grid, block, st, prm, cy)
+                   : launch_pdl(normtest_accumulate_kernel<BF16H, 1, 1, true>, grid, block, st, prm, cy);
+  } else if (dtype == ABS_F32) {
+    e = K <= 2   ? launch_pdl(normtest_accumulate_kernel<F32, 4, 2, false>, grid, block, st, prm, cy)
+        : K <= 4 ? launch_pdl(normtest_accumulate_kernel<F32, 2, 4, false>, grid, block, st, prm, cy)
+                 : launch_pdl(normtest_accumulate_kernel<F32, 1, 1, false>, grid, block, st, prm, cy);
+  } else {
+    e = K <= 4   ? launch_pdl(normtest_accumulate_kernel<BF16H, 4, 4, false>, grid, block, st, prm, cy)
+        : K <= 8 ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 8, false>, grid, block, st, prm, cy)
+                 : launch_pdl(normtest_accumulate_kernel<BF16H, 1, 1, false>, grid, block, st, prm, cy);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+
+  FinalizeParams fp;
+  std::memset(&fp, 0, sizeof fp);
+  fp.chunk_in = prm.chunk_out;
+  std::memcpy(fp.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
+  fp.n_shards = L.n_shards;
+  fp.n_chunks = L.n_chunks;
+  fp.stats = stats;
+  fp.b_next = b_next_out;
+  fp.eta = eta;
+  fp.norm = total;
+  fp.b_cur = b_cur;
+  std::memcpy(fp.shard_first, L.shard_off, sizeof(int64_t) * L.n_shards);
+  e = launch_finalize(fp, finalize_ctas, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return ABS_OK;
+}
+
 // Rows per row block of the per-sample kernels: at most 512 (the row-block records then cost
 // 1.6% of the matrix traffic), and, while the grid is only a few waves of 148 SMs x 3 resident
 // CTAs, the count that fills whole waves (b=4096, d=16384: 13 row blocks x 32 column blocks =
@@ -763,78 +875,22 @@ int abs_norm_test_accumulate(const void* const* grads, int K, int64_t d, abs_dty
                              const int64_t* shard_offsets, int n_shards, int64_t count_in,
                              double eta, int64_t b_cur, void* stats_inout, float* mean_inout,
                              int64_t* b_next_out, abs_stream_t stream) {
-  if (!grads || !stats_inout || !mean_inout || !b_next_out) return ABS_ERR_NULL;
-  if (dtype != ABS_F32 && dtype != ABS_BF16) return ABS_ERR_DTYPE;
-  if (K < 1 || K > kInlineWorkers || d < 1 || b_cur < 1) return ABS_ERR_RANGE;
-  if (count_in < 0 || count_in > (int64_t{1} << 40)) return ABS_ERR_RANGE;
-  if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
-  const size_t esz = (dtype == ABS_F32) ? 4 : 2;
-  for (int k = 0; k < K; ++k) {
-    if (!grads[k]) return ABS_ERR_NULL;
-    if (misaligned(grads[k], esz)) return ABS_ERR_ALIGN;
-  }
-  if (misaligned(stats_inout, 16) || misaligned(b_next_out, 8) || misaligned(mean_inout, 4))
-    return ABS_ERR_ALIGN;
-  Layout L;
-  const int rc = make_layout(d, shard_offsets, n_shards, false, &L);
-  if (rc != ABS_OK) return rc;
-  const size_t ud = static_cast<size_t>(d);
-  const Range outs[] = {{mean_inout, ud * 4}, {stats_inout, abs_stats_bytes(d, L.n_shards)},
-                        {b_next_out, 8}};
-  if (any_alias(grads, K, ud * esz, outs, 3)) return ABS_ERR_ALIAS;
-  const int finalize_ctas = finalize_max_cluster();
+  if (!mean_inout) return ABS_ERR_NULL;
+  return run_accumulate(grads, K, d, dtype, shard_offsets, n_shards, count_in, eta, b_cur,
+                        stats_inout, mean_inout, mean_inout, b_next_out, nullptr, nullptr, nullptr,
+                        nullptr, 0, false, stream);
+}
 
-  double* stats = static_cast<double*>(stats_inout);
-  StreamParams prm;
-  std::memset(&prm, 0, sizeof prm);
-  for (int k = 0; k < K; ++k) prm.grads[k] = grads[k];
-  std::memcpy(prm.shard_off, L.shard_off, sizeof(int64_t) * (L.n_shards + 1));
-  std::memcpy(prm.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
-  prm.d = d;
-  prm.K = K;
-  prm.n_shards = L.n_shards;
-  prm.n_chunks = L.n_chunks;
-  prm.chunk_elems = L.chunk_elems;
-  prm.gbar = mean_inout;
-  prm.chunk_out = stats + ABS_STATS_HEADER + static_cast<size_t>(L.n_shards) * ABS_SHARD_STRIDE;
-  const double total = static_cast<double>(count_in) + static_cast<double>(K);
-  AccumCarry cy;
-  cy.n_prev = static_cast<double>(count_in);
-  cy.inv_total = static_cast<float>(1.0 / total);
-  cy.shard_rec = stats + ABS_STATS_HEADER;
-
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const dim3 grid(static_cast<unsigned>(L.n_chunks)), block(kThreads);
-  cudaError_t e;
-  // few gradients per call: several thread-rows in flight per thread, 128 bytes of gradients
-  // either way (fp32: 16-byte vectors, bf16: 8-byte vectors)
-  if (dtype == ABS_F32) {
-    e = K <= 2   ? launch_pdl(normtest_accumulate_kernel<F32, 4, 2>, grid, block, st, prm, cy)
-        : K <= 4 ? launch_pdl(normtest_accumulate_kernel<F32, 2, 4>, grid, block, st, prm, cy)
-                 : launch_pdl(normtest_accumulate_kernel<F32, 1, 1>, grid, block, st, prm, cy);
-  } else {
-    // (eight rows for one or two bf16 gradients spill; four rows serve them)
-    e = K <= 4   ? launch_pdl(normtest_accumulate_kernel<BF16H, 4, 4>, grid, block, st, prm, cy)
-        : K <= 8 ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 8>, grid, block, st, prm, cy)
-                 : launch_pdl(normtest_accumulate_kernel<BF16H, 1, 1>, grid, block, st, prm, cy);
-  }
-  if (e != cudaSuccess) return cuda_fail(e);
-
-  FinalizeParams fp;
-  std::memset(&fp, 0, sizeof fp);
-  fp.chunk_in = prm.chunk_out;
-  std::memcpy(fp.chunk_prefix, L.chunk_prefix, sizeof(int32_t) * (L.n_shards + 1));
-  fp.n_shards = L.n_shards;
-  fp.n_chunks = L.n_chunks;
-  fp.stats = stats;
-  fp.b_next = b_next_out;
-  fp.eta = eta;
-  fp.norm = total;
-  fp.b_cur = b_cur;
-  std::memcpy(fp.shard_first, L.shard_off, sizeof(int64_t) * L.n_shards);
-  e = launch_finalize(fp, finalize_ctas, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-  return ABS_OK;
+int abs_norm_test_accumulate_adamw(const void* const* grads, int K, int64_t d, abs_dtype dtype,
+                                   const int64_t* shard_offsets, int n_shards, int64_t count_in,
+                                   double eta, int64_t b_cur, void* stats_inout,
+                                   const float* mean_in, float* gbar_out, int64_t* b_next_out,
+                                   float* params, float* m, float* v,
+                                   const abs_adamw_hparams* hparams, int64_t step,
+                                   abs_stream_t stream) {
+  return run_accumulate(grads, K, d, dtype, shard_offsets, n_shards, count_in, eta, b_cur,
+                        stats_inout, mean_in, gbar_out, b_next_out, params, m, v, hparams, step,
+                        true, stream);
 }
 
 int abs_noalloc_fits(int64_t d, const int64_t* shard_offsets, int n_shards) {

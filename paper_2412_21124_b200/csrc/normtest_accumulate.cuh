@@ -29,8 +29,12 @@ namespace absnt {
 struct AccumCarry {
   double n_prev;            // gradients merged by the earlier calls of this step; 0 starts a step
   float inv_total;          // 1 / (n_prev + K)
+  const float* mean_in;     // running mean of those n_prev gradients (unused when n_prev = 0)
   const double* shard_rec;  // shard records left by the previous call (slot 1: its sum S_s)
 };
+// The new mean goes to prm.gbar (which may be mean_in itself).  The closing call of a step can
+// run AdamW on it in the same pass (ADAM: prm.p, m, v, p16 as in the fused kernels); prm.gbar
+// may then be null -- the mean is consumed in registers and not written.
 
 // Accumulators of one thread-row (four coordinates as two packed pairs).
 template <typename GT>
@@ -90,7 +94,7 @@ struct AccumRow {
 
 // One thread-row with element-wise, bounds-checked accesses (ragged end of a shard, streams
 // that are not 16-byte aligned): the operations of AccumRow in the same order.
-template <typename GT>
+template <typename GT, bool ADAM>
 __device__ __noinline__ void accumulate_scalar_row(const StreamParams& prm, const AccumCarry& cy,
                                                    int K, int64_t base, int64_t hi, float* sums) {
   constexpr int H = split_group<GT, false>();
@@ -99,7 +103,7 @@ __device__ __noinline__ void accumulate_scalar_row(const StreamParams& prm, cons
   for (int e = 0; e < GT::kVec; ++e) {
     const int64_t i = base + e;
     if (i >= hi) break;
-    const float c = carry ? prm.gbar[i] : GT::load1(prm.grads[0], i);
+    const float c = carry ? cy.mean_in[i] : GT::load1(prm.grads[0], i);
     float s2 = 0.f, g2 = 0.f, sd = 0.f, gd = 0.f;
     for (int k = 0; k < K; ++k) {
       const float dv = GT::load1(prm.grads[k], i) - c;
@@ -115,7 +119,15 @@ __device__ __noinline__ void accumulate_scalar_row(const StreamParams& prm, cons
     const float mu = c + dm;
     row_n2 = fmaf(mu, mu, row_n2);
     row_S += clamp_nonneg(fmaf(-sd, dm, s2));
-    prm.gbar[i] = mu;
+    if (prm.gbar) prm.gbar[i] = mu;
+    if (ADAM) {
+      float w = prm.p[i], m = prm.m[i], v = prm.v[i];
+      adamw_elem(prm.adam, prm.adam.omb1, prm.adam.omb2, mu, w, m, v);
+      prm.p[i] = w;
+      prm.m[i] = m;
+      prm.v[i] = v;
+      if (prm.p16) prm.p16[i] = to_bf16(w);
+    }
   }
   sums[0] = row_n2;
   sums[1] = row_S;
@@ -125,8 +137,8 @@ __device__ __noinline__ void accumulate_scalar_row(const StreamParams& prm, cons
 // ROWS mean vectors: 128 bytes of gradients per thread for ROWS * KR = 8 vectors of 16 bytes or
 // 16 of 8 bytes) before the first is consumed; rows are consumed in order, so the sums have the
 // shape of the ROWS = 1 kernel and both give the same bits.
-template <typename GT, int ROWS, int KR>
-__global__ void __launch_bounds__(kThreads, 3)
+template <typename GT, int ROWS, int KR, bool ADAM>
+__global__ void __launch_bounds__(kThreads, ADAM ? 2 : 3)
     normtest_accumulate_kernel(const __grid_constant__ StreamParams prm,
                                const __grid_constant__ AccumCarry cy) {
   static_assert(GT::kVec == 4, "four coordinates per thread-row");
@@ -137,7 +149,9 @@ __global__ void __launch_bounds__(kThreads, 3)
   const int tid = threadIdx.x;
   const int chunk = blockIdx.x;
   const bool carry = cy.n_prev > 0.0;
-  const ChunkGeometry cg = chunk_geometry<GT, kInlineWorkers, false, false>(prm, prm.grads, K, chunk);
+  ChunkGeometry cg = chunk_geometry<GT, kInlineWorkers, false, ADAM>(prm, prm.grads, K, chunk);
+  if (carry && ((reinterpret_cast<uintptr_t>(cy.mean_in) + static_cast<uintptr_t>(cg.lo) * 4) & 15))
+    cg.aligned = false;
   // does this chunk open its shard?  (the shard: the last s with chunk_prefix[s] <= chunk)
   int lo_s = 0, hi_s = prm.n_shards;
   while (hi_s - lo_s > 1) {
@@ -153,18 +167,51 @@ __global__ void __launch_bounds__(kThreads, 3)
   auto vec_ptr = [&](int k, int64_t base) {
     return reinterpret_cast<const typename GT::scalar*>(prm.grads[k]) + base;
   };
+  struct State {
+    float4 w, m, v;
+  };
+  auto load_state = [&](int64_t base) {
+    State st;
+    if (ADAM) {
+      st.w = ld_state_16(prm.p + base);
+      st.m = ld_state_16(prm.m + base);
+      st.v = ld_state_16(prm.v + base);
+    }
+    return st;
+  };
+  // the row's new means: written, and (ADAM) consumed by the update of the row's parameters
+  auto finish_row = [&](AccumRow<GT>& acc, int64_t base, State& st) {
+    float row_n2 = 0.f, row_S = 0.f;
+    const float4 mu = acc.finish(cy.inv_total, row_n2, row_S);
+    if (prm.gbar) st_stream_16(prm.gbar + base, mu);
+    if (ADAM) {
+      float2* w2 = reinterpret_cast<float2*>(&st.w);
+      float2* m2 = reinterpret_cast<float2*>(&st.m);
+      float2* v2 = reinterpret_cast<float2*>(&st.v);
+      adamw_pair(prm.adam, prm.adam.omb1, prm.adam.omb2, make_float2(mu.x, mu.y), w2[0], m2[0], v2[0]);
+      adamw_pair(prm.adam, prm.adam.omb1, prm.adam.omb2, make_float2(mu.z, mu.w), w2[1], m2[1], v2[1]);
+      st_stream_16(prm.p + base, st.w);
+      st_stream_16(prm.m + base, st.m);
+      st_stream_16(prm.v + base, st.v);
+      if (prm.p16) st_bf16x4(prm.p16 + base, st.w);
+    }
+    acc_n2 += static_cast<double>(row_n2);
+    acc_S += static_cast<double>(row_S);
+  };
 
   if constexpr (ROWS > 1) {
     while (cg.aligned && row_lo + static_cast<int64_t>(ROWS) * kThreads * V <= hi) {
       typename GT::raw_t raw[ROWS][KR];
       float4 mo[ROWS];
+      State st[ROWS];
 #pragma unroll
       for (int r = 0; r < ROWS; ++r) {
         const int64_t base = row_lo + (static_cast<int64_t>(r) * kThreads + tid) * V;
 #pragma unroll
         for (int k = 0; k < KR; ++k)
           if (k < K) raw[r][k] = GT::load_vec(vec_ptr(k, base));
-        mo[r] = carry ? ld_state_16(prm.gbar + base) : make_float4(0.f, 0.f, 0.f, 0.f);
+        mo[r] = carry ? ld_state_16(cy.mean_in + base) : make_float4(0.f, 0.f, 0.f, 0.f);
+        st[r] = load_state(base);
       }
 #pragma unroll
       for (int r = 0; r < ROWS; ++r) {
@@ -175,10 +222,7 @@ __global__ void __launch_bounds__(kThreads, 3)
         for (int k = 0; k < KR; ++k)
           if (k < K) acc.add(raw[r][k]);
         acc.close_group();
-        float row_n2 = 0.f, row_S = 0.f;
-        st_stream_16(prm.gbar + base, acc.finish(cy.inv_total, row_n2, row_S));
-        acc_n2 += static_cast<double>(row_n2);
-        acc_S += static_cast<double>(row_S);
+        finish_row(acc, base, st[r]);
       }
       row_lo += static_cast<int64_t>(ROWS) * kThreads * V;
     }
@@ -186,11 +230,11 @@ __global__ void __launch_bounds__(kThreads, 3)
 
   for (; row_lo < hi; row_lo += kThreads * V) {
     const int64_t base = row_lo + static_cast<int64_t>(tid) * V;
-    float row_n2 = 0.f, row_S = 0.f;
     if (cg.aligned && row_lo + kThreads * V <= hi) {
       AccumRow<GT> acc;
       bool need_centre = !carry;  // uniform across the CTA
-      if (carry) acc.init(ld_state_16(prm.gbar + base));
+      if (carry) acc.init(ld_state_16(cy.mean_in + base));
+      State st = load_state(base);  // in flight while the gradients are consumed
       // N consecutive workers from k0: all loads first, then the arithmetic
       auto piece = [&](int k0, auto n_tag) {
         constexpr int N = decltype(n_tag)::value;
@@ -224,15 +268,13 @@ __global__ void __launch_bounds__(kThreads, 3)
       }
       if ((K - k0) & 1) piece(k0, std::integral_constant<int, 1>{});
       acc.close_group();  // adds exact zeros when K is a multiple of H
-      st_stream_16(prm.gbar + base, acc.finish(cy.inv_total, row_n2, row_S));
+      finish_row(acc, base, st);
     } else if (base < hi) {
       float sums[2];
-      accumulate_scalar_row<GT>(prm, cy, K, base, hi, sums);
-      row_n2 = sums[0];
-      row_S = sums[1];
+      accumulate_scalar_row<GT, ADAM>(prm, cy, K, base, hi, sums);
+      acc_n2 += static_cast<double>(sums[0]);
+      acc_S += static_cast<double>(sums[1]);
     }
-    acc_n2 += static_cast<double>(row_n2);
-    acc_S += static_cast<double>(row_S);
   }
   // the shard's sum so far rides on the first thread's partial of the shard's first chunk
   if (carry && opens_shard && tid == 0)

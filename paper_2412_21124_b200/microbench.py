@@ -50,6 +50,8 @@ def bytes_per_call(call, d, K, esz, gbar, b):
         return 28 * d
     if call == "accumulate":  # the K new gradients once, the running mean read and written
         return (K * esz + 8) * d
+    if call == "accumulate_adamw":  # the closing call: mean read, p/m/v read and written
+        return (K * esz + 4 + 24) * d
     return esz * b * d
 
 
@@ -67,14 +69,14 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
     sets = []
     for i in range(n_sets):
         s = {}
-        if call in ("fused", "normtest", "accumulate"):
+        if call in ("fused", "normtest", "accumulate", "accumulate_adamw"):
             sizes = _sizes(d)
             sig = synth.per_tensor_sigma(sizes, 11)
             s["grads"] = synth.worker_grads(sizes, K, tdt, 100 + i, dev, sigma=sig)
             s["stats"] = B.alloc_stats(d, n_shards, dev)
-        if call in ("fused", "adamw"):
+        if call in ("fused", "adamw", "accumulate_adamw"):
             s["p"], s["m"], s["v"] = synth.adam_state(d, 200 + i, dev, zero_moments=False)
-        if call in ("normtest", "adamw", "accumulate") or gbar:
+        if call in ("normtest", "adamw", "accumulate", "accumulate_adamw") or gbar:
             s["gbar"] = torch.zeros(d, dtype=torch.float32, device=dev)
             if call == "adamw":
                 s["gbar"].normal_().mul_(0.02)
@@ -106,6 +108,10 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
         elif call == "accumulate":  # a later call of a step: the running mean is read and written
             B.abs_norm_test_accumulate(s["grads"], 8 * K, 0.1, 512, s["stats"], s["gbar"],
                                        s["b_next"], shard_offsets=offs)
+        elif call == "accumulate_adamw":  # the closing call of a step, the mean not written
+            B.abs_norm_test_accumulate_adamw(s["grads"], 8 * K, 0.1, 512, s["stats"], s["gbar"],
+                                             None, s["b_next"], s["p"], s["m"], s["v"], HP,
+                                             100 + i, shard_offsets=offs)
         else:
             B.abs_persample_norm_test(s["G"], 0.1, s["stats"], s["gbar"], s["b_next"])
 
@@ -200,6 +206,7 @@ REPORT_POINTS = (
        ("fused", GPT2, 32, "bf16", 1, {"coordwise": True})]
     # the carry-in form: K new gradients merged into the running mean per call
     + [("accumulate", GPT2, K, dt, 1, {}) for K in (1, 2, 4, 8, 16) for dt in ("bf16", "f32")]
+    + [("accumulate_adamw", GPT2, K, "bf16", 1, {}) for K in (1, 4, 8)]
     # the paper's own model sizes (Table 4), J = 4 workers, bf16
     + [("fused", d, 4, "bf16", 1, {}) for d in (304_600_000, 1_100_000_000, 3_400_000_000)])
 
@@ -282,7 +289,8 @@ def format_markdown(path):
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("--call", choices=["fused", "normtest", "adamw", "persample", "accumulate"], default="fused")
+    ap.add_argument("--call", choices=["fused", "normtest", "adamw", "persample", "accumulate",
+                                       "accumulate_adamw"], default="fused")
     ap.add_argument("--d", type=int, default=33_554_432)
     ap.add_argument("--K", type=int, default=8)
     ap.add_argument("--dtype", choices=["bf16", "f32"], default="bf16")

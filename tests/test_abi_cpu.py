@@ -299,6 +299,32 @@ def test_accumulate_rejects(L, over, status):
     assert L.abs_norm_test_accumulate(*_acc_args(**over)) == status
 
 
+def test_accumulate_adamw_rejects(L):
+    hp = binding.abs_adamw_hparams(1e-3, 0.9, 0.999, 1e-8, 0.1)
+    far = [FAKE + i * 0x100000 for i in range(1, 12)]
+    table = (ctypes.c_void_p * 4)(far[0], far[1])
+
+    def call(**over):
+        a = dict(grads=table, K=2, d=100, dtype=0, offs=None, n_shards=1, count_in=3, eta=0.1,
+                 b_cur=8, stats=far[2], mean=far[3], gbar=far[3], b_next=far[4], p=far[5], m=far[6],
+                 v=far[7], hp=ctypes.byref(hp), step=1, stream=None)
+        a.update(over)
+        return L.abs_norm_test_accumulate_adamw(*[a[k] for k in (
+            "grads", "K", "d", "dtype", "offs", "n_shards", "count_in", "eta", "b_cur", "stats",
+            "mean", "gbar", "b_next", "p", "m", "v", "hp", "step", "stream")])
+
+    assert call(mean=None) == binding.ABS_ERR_NULL            # a running step needs its mean
+    assert call(p=None) == binding.ABS_ERR_NULL
+    assert call(hp=None) == binding.ABS_ERR_NULL
+    assert call(step=0) == binding.ABS_ERR_RANGE
+    assert call(K=65) == binding.ABS_ERR_RANGE
+    assert call(m=far[6] + 2) == binding.ABS_ERR_ALIGN
+    assert call(gbar=far[3] + 16) == binding.ABS_ERR_ALIAS     # overlaps the mean without being it
+    assert call(gbar=far[5]) == binding.ABS_ERR_ALIAS          # the mean output on the parameters
+    assert call(mean=far[6]) == binding.ABS_ERR_ALIAS          # the running mean on a moment
+    assert call(v=far[0] + 8) == binding.ABS_ERR_ALIAS         # an output on a gradient buffer
+
+
 def _hp(**over):
     v = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
     v.update(over)

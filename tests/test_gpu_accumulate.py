@@ -16,12 +16,14 @@ import torch
 import paper_2412_21124_b200 as absnt
 from oracle import abs_oracle as orc
 from paper_2412_21124_b200 import synth
-from tests.util import REL_VEC, assert_sum_close, assert_vec_close, margin_ok, to_host
+from tests.util import (REL_VEC, assert_sum_close, assert_vec_close, margin_ok, oracle_adamw,
+                        to_host)
 
 pytestmark = pytest.mark.gpu
 
 DEV = "cuda:0"
 D = 4 * 4096 + 1234   # several chunks of 4096 and a ragged tail
+HP = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -233,3 +235,102 @@ def test_accumulate_config2_size_sampled():
                      b_cur):
             break
     accumulate_and_check(grads, [1] * K, eta, b_cur, check_every_call=False)
+
+
+# ------------------------------------------------------------- closing call fused with AdamW
+CLOSING = [([8], "whole step"), ([7, 1], "one"), ([4, 4], "two rows"), ([3, 9], "general"),
+           ([1] * 5, "micro-batches"), ([20, 33], "groups")]
+
+
+@pytest.mark.parametrize("inplace", [True, False], ids=["mean in place", "mean not written"])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("parts", [c[0] for c in CLOSING], ids=[c[1] for c in CLOSING])
+def test_accumulate_closing_call_with_adamw(parts, dtype, inplace):
+    """All calls but the last merge; the last one merges and applies AdamW with the final mean
+    (Algorithm 1: the test, then the update on the batch gradient).  Sums, decision, parameters
+    and moments against the oracle's plain test + AdamW on all buffers."""
+    K, eta, b_cur, step = sum(parts), 0.1, 64, 4
+    seed = 500 + K
+    while True:
+        grads = synth.worker_grads([D], K, dtype, seed, DEV)
+        ref = orc.norm_test([to_host(g) for g in grads], eta, b_cur)
+        if margin_ok(ref["T"], b_cur):
+            break
+        seed += 1
+    p, m, v = synth.adam_state(D, 12, DEV, zero_moments=False)
+    p0, m0, v0 = to_host(p), to_host(m), to_host(v)
+    stats = absnt.alloc_stats(D, 1, DEV)
+    mean = torch.zeros(D, dtype=torch.float32, device=DEV)
+    b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+    count = 0
+    for mpart in parts[:-1]:
+        absnt.abs_norm_test_accumulate(grads[count:count + mpart], count, eta, b_cur, stats, mean,
+                                       b_next)
+        count += mpart
+    before = mean.clone()
+    absnt.abs_norm_test_accumulate_adamw(grads[count:], count, eta, b_cur, stats,
+                                         mean if count else None, mean if inplace else None,
+                                         b_next, p, m, v, HP, step)
+    torch.cuda.synchronize()
+    got = absnt.read_stats(stats)
+    assert got["norm"] == K
+    assert_sum_close(got["n2"], ref["n2"], "n2")
+    assert_sum_close(got["S"], ref["S"], "S")
+    assert int(b_next.item()) == ref["b_next"] and got["flags"] == ref["flags"]
+    if inplace:
+        assert_vec_close(mean, ref["gbar"], "final mean", rel=mean_tolerance(len(parts)))
+    else:
+        assert torch.equal(mean, before)   # the running mean was only read
+    w_ref, m_ref, v_ref = oracle_adamw(orc, p0, m0, v0, ref["gbar"], HP, step)
+    assert_vec_close(p, w_ref, "params")
+    assert_vec_close(m, m_ref, "m")
+    assert_vec_close(v, v_ref, "v")
+
+
+def test_accumulate_closing_call_equals_merge_then_adamw():
+    """The fused closing call against the two-call form (abs_norm_test_accumulate, then
+    abs_adamw_step on the final mean): the same mean, sums and decision bit for bit, and the
+    same update (both run adamw on the same fp32 mean)."""
+    K = 6
+    grads = synth.worker_grads([D], K, torch.bfloat16, 77, DEV)
+    outs = []
+    for fused in (False, True):
+        p, m, v = synth.adam_state(D, 13, DEV, zero_moments=False)
+        stats = absnt.alloc_stats(D, 1, DEV)
+        mean = torch.zeros(D, dtype=torch.float32, device=DEV)
+        b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+        absnt.abs_norm_test_accumulate(grads[:4], 0, 0.1, 64, stats, mean, b_next)
+        if fused:
+            absnt.abs_norm_test_accumulate_adamw(grads[4:], 4, 0.1, 64, stats, mean, mean, b_next,
+                                                 p, m, v, HP, 9)
+        else:
+            absnt.abs_norm_test_accumulate(grads[4:], 4, 0.1, 64, stats, mean, b_next)
+            absnt.abs_adamw_step(p, mean, m, v, HP, 9)
+        torch.cuda.synchronize()
+        outs.append((absnt.read_stats(stats), mean, int(b_next.item()), p, m, v))
+    a, b = outs
+    for key in ("n2", "S", "T", "flags"):
+        assert a[0][key] == b[0][key], key
+    assert a[2] == b[2]
+    for x, y in zip(a[1:2] + a[3:], b[1:2] + b[3:]):
+        assert torch.equal(x, y)
+
+
+def test_accumulate_adamw_misaligned_and_ragged():
+    """State vectors that are not 16-byte aligned take the element-wise path of the fused
+    closing call: the same bits as the aligned run."""
+    grads = synth.worker_grads([D], 5, torch.float32, 61, DEV)
+    res = []
+    for shift in (0, 1):
+        p, m, v = (shifted_copy(t, shift) for t in synth.adam_state(D, 14, DEV, zero_moments=False))
+        stats = absnt.alloc_stats(D, 1, DEV)
+        mean = shifted_copy(torch.zeros(D, dtype=torch.float32, device=DEV), shift)
+        b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+        absnt.abs_norm_test_accumulate(grads[:2], 0, 0.1, 64, stats, mean, b_next)
+        absnt.abs_norm_test_accumulate_adamw(grads[2:], 2, 0.1, 64, stats, mean, mean, b_next,
+                                             p, m, v, HP, 2)
+        torch.cuda.synchronize()
+        res.append((absnt.read_stats(stats)["S"], mean.clone(), p.clone(), m.clone(), v.clone()))
+    assert res[0][0] == res[1][0]
+    for x, y in zip(res[0][1:], res[1][1:]):
+        assert torch.equal(x, y)
