@@ -472,8 +472,8 @@ int run_accumulate(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   const dim3 grid(static_cast<unsigned>(L.n_chunks)), block(kThreads);
   cudaError_t e;
   // few gradients per call: several thread-rows in flight per thread, 128 bytes of gradients
-  // either way (fp32: 16-byte vectors, bf16: 8-byte vectors; eight rows for one or two bf16
-  // gradients spill, four rows serve them).  With AdamW the state vectors are in flight as
+  // either way (fp32: 16-byte vectors, bf16: 8-byte vectors; eight rows fit for a single bf16
+  // gradient and spill otherwise).  With AdamW the state vectors are in flight as
   // well: two rows up to four gradients, one beyond.
   if (fused) {
     if (dtype == ABS_F32)
@@ -488,7 +488,8 @@ int run_accumulate(const void* const* grads, int K, int64_t d, abs_dtype dtype,
         : K <= 4 ? launch_pdl(normtest_accumulate_kernel<F32, 2, 4, false>, grid, block, st, prm, cy)
                  : launch_pdl(normtest_accumulate_kernel<F32, 1, 1, false>, grid, block, st, prm, cy);
   } else {
-    e = K <= 4   ? launch_pdl(normtest_accumulate_kernel<BF16H, 4, 4, false>, grid, block, st, prm, cy)
+    e = K == 1   ? launch_pdl(normtest_accumulate_kernel<BF16H, 8, 1, false>, grid, block, st, prm, cy)
+        : K <= 4 ? launch_pdl(normtest_accumulate_kernel<BF16H, 4, 4, false>, grid, block, st, prm, cy)
         : K <= 8 ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 8, false>, grid, block, st, prm, cy)
                  : launch_pdl(normtest_accumulate_kernel<BF16H, 1, 1, false>, grid, block, st, prm, cy);
   }
