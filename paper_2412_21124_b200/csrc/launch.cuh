@@ -81,16 +81,13 @@ cudaError_t launch_one(const StreamParams& prm, cudaStream_t st) {
   // Measured exceptions.  Fused: the 512-coordinate tile loses to the register-direct kernel
   // when the worker loop is predicated (EXACT false; K=12: 5.46 vs 5.80 TB/s).  Unfused test
   // (K*s + 4 bytes per coordinate, so more coordinates per second and more instructions per
-  // byte): staging wins by 1-9% for most worker counts (fp32 K=5 6.39 -> 6.96 TB/s, bf16 K=9
-  // 6.42 -> 6.87) but loses where the register-direct kernel is at its best: one or two
-  // workers (bf16 K=1 -37%, K=2 -7%; fp32 K=2 equal) and bf16 K=6 (-0.4%).  bf16 K=8: with the
-  // diagnostic Q computed the staged kernel loses 2.8%; without it the two are equal at
-  // d = 124M and staging wins at 1.24G coordinates in 8 shards (6.78 -> 6.90 TB/s), so the
-  // plain test stages it.
+  // byte): staging wins for every worker count from 3 up (by 1-9%; with three resident CTAs,
+  // see bulk_shape, also for bf16 K=6 and for K=8 with the diagnostic Q or the coordinate-wise
+  // maximum, which two CTAs had left to the register-direct kernel) and loses for one or two
+  // workers, where the register-direct kernel is at its best (bf16 K=1 -37%, K=2 -1%; fp32 K=2
+  // equal).
   constexpr BulkShape shape = bulk_shape<GT, KB, ADAM>();
-  constexpr bool kBf16 = std::is_same<GT, BF16>::value;
-  constexpr bool staged_test =
-      EXACT && KB >= 3 && !(kBf16 && (KB == 6 || (KB == 8 && STAT != kStatSums)));
+  constexpr bool staged_test = EXACT && KB >= 3;
   constexpr int tile = ADAM ? ((shape.tile == 512 && !EXACT) ? 0 : shape.tile)
                             : (staged_test ? shape.tile : 0);
   if constexpr (tile > 0) {

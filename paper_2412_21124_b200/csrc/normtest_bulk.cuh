@@ -44,6 +44,17 @@ struct BulkShape {
 };
 template <typename GT, int KB, bool ADAM>
 __host__ __device__ constexpr BulkShape bulk_shape() {
+  // The test alone has small stages (no optimizer state), so three CTAs of three or more
+  // stages fit for up to 10 bf16 / 4 fp32 workers: 24 warps per SM instead of 16 cover the
+  // per-tile barrier and the wait for a tile's arrival better (bf16 K=7 6.64 -> 6.91 TB/s, K=8
+  // 6.70 -> 6.88, K=9, 10 +3%; fp32 K=3 6.65 -> 6.91; K=8 bf16 on 1.24G coordinates in 8 shards
+  // 6.88 -> 7.11; bf16 K=6, which used to prefer the register-direct kernel, 6.64 -> 6.95; nothing
+  // lost for K = 3..5).
+  // The fused kernels with stages small enough for this (bf16 K <= 4, fp32 K <= 2) lose 0.4-0.9%.
+  if (!ADAM && 3 * 3 * bulk_stage_bytes<GT, KB, ADAM>(1024) <= kSmemPerSM) {
+    const int fit = kSmemPerSM / (3 * bulk_stage_bytes<GT, KB, ADAM>(1024));
+    return {1024, fit > 5 ? 5 : fit, 3};
+  }
   if (2 * 3 * bulk_stage_bytes<GT, KB, ADAM>(1024) <= kSmemPerSM) {
     // small stages (few workers): up to five of them, so that as many bytes stay in flight
     const int fit = kSmemPerSM / (2 * bulk_stage_bytes<GT, KB, ADAM>(1024));
