@@ -45,7 +45,7 @@ struct BulkShape {
 template <typename GT, int KB, bool ADAM>
 __host__ __device__ constexpr BulkShape bulk_shape() {
   // The test alone has small stages (no optimizer state), so three CTAs of three or more
-  // stages fit for up to 10 bf16 / 4 fp32 workers: 24 warps per SM instead of 16 cover the
+  // stages fit for up to 10 bf16 / 5 fp32 workers: 24 warps per SM instead of 16 cover the
   // per-tile barrier and the wait for a tile's arrival better (bf16 K=7 6.64 -> 6.91 TB/s, K=8
   // 6.70 -> 6.88, K=9, 10 +3%; fp32 K=3 6.65 -> 6.91; K=8 bf16 on 1.24G coordinates in 8 shards
   // 6.88 -> 7.11; bf16 K=6, which used to prefer the register-direct kernel, 6.64 -> 6.95; nothing
