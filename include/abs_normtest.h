@@ -373,6 +373,21 @@ int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs
                             abs_stream_t stream);
 
 /*
+ * The coordinate-wise test in its per-sample form (Sec. 4, Proposition 1: the condition is asked
+ * of every coordinate, with the per-sample variance of that coordinate): the same pass over G,
+ * the same gbar, n2 and S, but
+ *   T_i = (sum_r (G[r,i]-gbar_i)^2 / (b-1)) / (eta^2 gbar_i^2),   T = max_i T_i
+ * (T_i = 0 where the column has zero variance, +inf where only gbar_i = 0: then the test fails
+ * for every batch size and b_next saturates, flag DEGENERATE).  The header's T slot holds T, its
+ * ARGMAX slot the column where it occurs (the lowest one on a tie), the shard record is
+ * {n2, S, that column, T}.  Arguments and the zero-filled stats buffer as for
+ * abs_persample_norm_test.
+ */
+int abs_persample_norm_test_coordwise(const void* G, int64_t b, int64_t d, int64_t ld,
+                                      abs_dtype dtype, double eta, void* stats_out,
+                                      float* gbar_out, int64_t* b_next_out, abs_stream_t stream);
+
+/*
  * The decision alone, on the host, from sums already reduced (e.g. to re-decide for a
  * different eta, or after combining per-rank sums in rank order).  Same expression
  * order as the device code: T = (S/norm) / ((eta*eta)*n2).  Writes T and the ABS_FLAG_*

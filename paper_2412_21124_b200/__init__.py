@@ -11,7 +11,7 @@ from .binding import (ABS_BF16, ABS_F32, ABS_FLAG_DEGENERATE, ABS_FLAG_NONFINITE
                       abs_norm_test_coordwise, abs_normtest_adamw_coordwise, abs_norm_test_q,
                       abs_norm_test_accumulate, abs_norm_test_accumulate_adamw,
                       abs_normtest_adamw_clip_prev, abs_selftest_bounded_wait,
-                      abs_persample_norm_test,
+                      abs_persample_norm_test, abs_persample_norm_test_coordwise,
                       abs_persample_stats_bytes, abs_round_batch, abs_schedule_advance,
                       abs_schedule_init, abs_schedule_test_due, abs_stats_bytes,
                       alloc_persample_stats, alloc_stats, read_stats)

@@ -94,6 +94,8 @@ def lib():
     L.abs_adamw_step_mixed.argtypes = [ptr, ptr, ptr, ptr, ptr, i64, ptr, i64, dbl, ptr, ptr]
     L.abs_persample_norm_test.restype = cint
     L.abs_persample_norm_test.argtypes = [ptr, i64, i64, i64, cint, dbl, ptr, ptr, ptr, ptr]
+    L.abs_persample_norm_test_coordwise.restype = cint
+    L.abs_persample_norm_test_coordwise.argtypes = list(L.abs_persample_norm_test.argtypes)
     L.abs_noalloc_fits.restype = cint
     L.abs_noalloc_fits.argtypes = [i64, ptr, cint]
     L.abs_combine_sums.restype = i64
@@ -536,7 +538,8 @@ class FusedStep:
             raise AbsError(rc, "abs_normtest_adamw")
 
 
-def abs_persample_norm_test(G, eta, stats_out, gbar_out, b_next_out, stream=None):
+def abs_persample_norm_test(G, eta, stats_out, gbar_out, b_next_out, stream=None,
+                            _entry="abs_persample_norm_test"):
     if G.dim() != 2 or G.stride(1) != 1 or not G.is_cuda:
         raise TypeError("G must be a CUDA matrix [b, d] with unit column stride")
     b, d, ld = G.shape[0], G.shape[1], G.stride(0)
@@ -544,11 +547,18 @@ def abs_persample_norm_test(G, eta, stats_out, gbar_out, b_next_out, stream=None
     _check_stats(stats_out, abs_persample_stats_bytes(b, d))
     _check_b_next(b_next_out)
     _check_one_device(G, stats_out, gbar_out, b_next_out)
-    rc = lib().abs_persample_norm_test(G.data_ptr(), b, d, ld, _dtype_code(G), float(eta),
-                                       stats_out.data_ptr(), gbar_out.data_ptr(),
-                                       b_next_out.data_ptr(), _stream(stream))
+    rc = getattr(lib(), _entry)(G.data_ptr(), b, d, ld, _dtype_code(G), float(eta),
+                                stats_out.data_ptr(), gbar_out.data_ptr(),
+                                b_next_out.data_ptr(), _stream(stream))
     if rc != ABS_OK:
-        raise AbsError(rc, "abs_persample_norm_test")
+        raise AbsError(rc, _entry)
+
+
+def abs_persample_norm_test_coordwise(G, eta, stats_out, gbar_out, b_next_out, stream=None):
+    """The per-sample call with the coordinate-wise test as its decision (T = max over columns,
+    the column in the ABS_STAT_ARGMAX slot)."""
+    abs_persample_norm_test(G, eta, stats_out, gbar_out, b_next_out, stream,
+                            _entry="abs_persample_norm_test_coordwise")
 
 
 def abs_decide(S, n2, norm, eta, b_cur):

@@ -540,6 +540,72 @@ int persample_rows_per_block(int64_t b, int64_t d) {
   return static_cast<int>(rpb < INT32_MAX ? rpb : INT32_MAX);
 }
 
+// The one body behind abs_persample_norm_test and its coordinate-wise form.
+int run_persample(const void* G, int64_t b, int64_t d, int64_t ld, abs_dtype dtype, double eta,
+                  void* stats_out, float* gbar_out, int64_t* b_next_out, bool coordwise,
+                  abs_stream_t stream) {
+  if (!G || !stats_out || !gbar_out || !b_next_out) return ABS_ERR_NULL;
+  if (dtype != ABS_F32 && dtype != ABS_BF16) return ABS_ERR_DTYPE;
+  if (b < 2 || d < 1 || ld < d) return ABS_ERR_RANGE;
+  if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
+  const size_t esz = (dtype == ABS_F32) ? 4 : 2;
+  if (misaligned(G, esz) || misaligned(gbar_out, 4) || misaligned(stats_out, 16) ||
+      misaligned(b_next_out, 8))
+    return ABS_ERR_ALIGN;
+  const int64_t ncb = persample_col_blocks(d);
+  const int rpb = persample_rows_per_block(b, d);
+  const int64_t nrb = (b + rpb - 1) / rpb;
+  if (ncb > INT32_MAX || nrb > 65535) return ABS_ERR_RANGE;
+  if (overlaps(G, (static_cast<size_t>(b - 1) * ld + static_cast<size_t>(d)) * esz, gbar_out,
+               static_cast<size_t>(d) * 4))
+    return ABS_ERR_ALIAS;
+
+  double* stats = static_cast<double*>(stats_out);
+  PersampleParams prm;
+  std::memset(&prm, 0, sizeof prm);
+  prm.G = G;
+  prm.b = b;
+  prm.d = d;
+  prm.ld = ld;
+  prm.rows_per_block = rpb;
+  prm.n_row_blocks = static_cast<int>(nrb);
+  const int64_t nmb = (d + kPsThreads - 1) / kPsThreads;  // CTAs of the merge pass
+  if (nmb > INT32_MAX) return ABS_ERR_RANGE;
+  // the ticket counter sits at the same place whatever b and d are, so a buffer that has
+  // served one shape (and therefore holds zero there) serves any other shape it is large enough for
+  prm.tickets = reinterpret_cast<unsigned int*>(stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE);
+  prm.cb_rec = stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE + kPsTicketDoubles;
+  prm.ws_sum = prm.cb_rec + kPsRecDoubles * nmb;
+  prm.ws_m2 = prm.ws_sum + nrb * d;
+  prm.gbar = gbar_out;
+  prm.stats = stats;
+  prm.b_next = b_next_out;
+  prm.eta = eta;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // rows that start on a vector boundary (16 bytes of fp32, 8 of bf16) go through the
+  // asynchronous-copy ring; anything else takes element loads with the same arithmetic
+  const size_t vec_bytes = 4 * esz;
+  const bool ring = !misaligned(G, vec_bytes) && ((ld * esz) % vec_bytes == 0);
+  const dim3 grid(static_cast<unsigned>(ncb), static_cast<unsigned>(nrb));
+  const size_t ring_bytes = static_cast<size_t>(kRing) * kPsThreads * vec_bytes;
+  cudaError_t e;
+  if (dtype == ABS_F32)
+    e = ring ? launch_pdl_smem(persample_partial_kernel<PsF32, true>, grid, dim3(kPsThreads), ring_bytes,
+                               st, prm)
+             : launch_pdl(persample_partial_kernel<PsF32, false>, grid, dim3(kPsThreads), st, prm);
+  else
+    e = ring ? launch_pdl_smem(persample_partial_kernel<PsBF16, true>, grid, dim3(kPsThreads), ring_bytes,
+                               st, prm)
+             : launch_pdl(persample_partial_kernel<PsBF16, false>, grid, dim3(kPsThreads), st, prm);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const dim3 merge_grid(static_cast<unsigned>(nmb));
+  e = coordwise ? launch_pdl(persample_merge_kernel<true>, merge_grid, dim3(kPsThreads), st, prm)
+                : launch_pdl(persample_merge_kernel<false>, merge_grid, dim3(kPsThreads), st, prm);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return ABS_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -559,7 +625,7 @@ size_t abs_persample_stats_bytes(int64_t b, int64_t d) {
   const size_t nmb = static_cast<size_t>((d + kPsThreads - 1) / kPsThreads);
   // header, one shard record, the ticket counter (two doubles' worth, at a fixed place),
   // {n2, S} per CTA of the merge pass, {sum, M2} per (row block, column)
-  return sizeof(double) * (ABS_STATS_HEADER + ABS_SHARD_STRIDE + kPsTicketDoubles + 2 * nmb +
+  return sizeof(double) * (ABS_STATS_HEADER + ABS_SHARD_STRIDE + kPsTicketDoubles + kPsRecDoubles * nmb +
                            2 * nrb * static_cast<size_t>(d));
 }
 
@@ -736,65 +802,13 @@ int abs_adamw_step_mixed(float* params, const float* gbar, float* m, float* v,
 int abs_persample_norm_test(const void* G, int64_t b, int64_t d, int64_t ld, abs_dtype dtype,
                             double eta, void* stats_out, float* gbar_out, int64_t* b_next_out,
                             abs_stream_t stream) {
-  if (!G || !stats_out || !gbar_out || !b_next_out) return ABS_ERR_NULL;
-  if (dtype != ABS_F32 && dtype != ABS_BF16) return ABS_ERR_DTYPE;
-  if (b < 2 || d < 1 || ld < d) return ABS_ERR_RANGE;
-  if (!std::isfinite(eta) || !(eta > 0.0)) return ABS_ERR_RANGE;
-  const size_t esz = (dtype == ABS_F32) ? 4 : 2;
-  if (misaligned(G, esz) || misaligned(gbar_out, 4) || misaligned(stats_out, 16) ||
-      misaligned(b_next_out, 8))
-    return ABS_ERR_ALIGN;
-  const int64_t ncb = persample_col_blocks(d);
-  const int rpb = persample_rows_per_block(b, d);
-  const int64_t nrb = (b + rpb - 1) / rpb;
-  if (ncb > INT32_MAX || nrb > 65535) return ABS_ERR_RANGE;
-  if (overlaps(G, (static_cast<size_t>(b - 1) * ld + static_cast<size_t>(d)) * esz, gbar_out,
-               static_cast<size_t>(d) * 4))
-    return ABS_ERR_ALIAS;
+  return run_persample(G, b, d, ld, dtype, eta, stats_out, gbar_out, b_next_out, false, stream);
+}
 
-  double* stats = static_cast<double*>(stats_out);
-  PersampleParams prm;
-  std::memset(&prm, 0, sizeof prm);
-  prm.G = G;
-  prm.b = b;
-  prm.d = d;
-  prm.ld = ld;
-  prm.rows_per_block = rpb;
-  prm.n_row_blocks = static_cast<int>(nrb);
-  const int64_t nmb = (d + kPsThreads - 1) / kPsThreads;  // CTAs of the merge pass
-  if (nmb > INT32_MAX) return ABS_ERR_RANGE;
-  // the ticket counter sits at the same place whatever b and d are, so a buffer that has
-  // served one shape (and therefore holds zero there) serves any other shape it is large enough for
-  prm.tickets = reinterpret_cast<unsigned int*>(stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE);
-  prm.cb_rec = stats + ABS_STATS_HEADER + ABS_SHARD_STRIDE + kPsTicketDoubles;
-  prm.ws_sum = prm.cb_rec + 2 * nmb;
-  prm.ws_m2 = prm.ws_sum + nrb * d;
-  prm.gbar = gbar_out;
-  prm.stats = stats;
-  prm.b_next = b_next_out;
-  prm.eta = eta;
-
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // rows that start on a vector boundary (16 bytes of fp32, 8 of bf16) go through the
-  // asynchronous-copy ring; anything else takes element loads with the same arithmetic
-  const size_t vec_bytes = 4 * esz;
-  const bool ring = !misaligned(G, vec_bytes) && ((ld * esz) % vec_bytes == 0);
-  const dim3 grid(static_cast<unsigned>(ncb), static_cast<unsigned>(nrb));
-  const size_t ring_bytes = static_cast<size_t>(kRing) * kPsThreads * vec_bytes;
-  cudaError_t e;
-  if (dtype == ABS_F32)
-    e = ring ? launch_pdl_smem(persample_partial_kernel<PsF32, true>, grid, dim3(kPsThreads), ring_bytes,
-                               st, prm)
-             : launch_pdl(persample_partial_kernel<PsF32, false>, grid, dim3(kPsThreads), st, prm);
-  else
-    e = ring ? launch_pdl_smem(persample_partial_kernel<PsBF16, true>, grid, dim3(kPsThreads), ring_bytes,
-                               st, prm)
-             : launch_pdl(persample_partial_kernel<PsBF16, false>, grid, dim3(kPsThreads), st, prm);
-  if (e != cudaSuccess) return cuda_fail(e);
-  e = launch_pdl(persample_merge_kernel, dim3(static_cast<unsigned>(nmb)), dim3(kPsThreads), st,
-                 prm);
-  if (e != cudaSuccess) return cuda_fail(e);
-  return ABS_OK;
+int abs_persample_norm_test_coordwise(const void* G, int64_t b, int64_t d, int64_t ld,
+                                      abs_dtype dtype, double eta, void* stats_out,
+                                      float* gbar_out, int64_t* b_next_out, abs_stream_t stream) {
+  return run_persample(G, b, d, ld, dtype, eta, stats_out, gbar_out, b_next_out, true, stream);
 }
 
 int64_t abs_decide(double S, double n2, double norm, double eta, int64_t b_cur, double* T_out,

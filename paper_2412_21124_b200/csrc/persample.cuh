@@ -38,7 +38,7 @@
 #pragma once
 #include <type_traits>
 
-#include "abs_device.cuh"
+#include "normtest_stream.cuh"
 
 namespace absnt {
 
@@ -68,7 +68,8 @@ struct PersampleParams {
   double* ws_sum;  // [n_row_blocks][d]
   double* ws_m2;
   float* gbar;
-  double* cb_rec;         // 2 doubles {n2, S} per CTA of pass 2 (kPsThreads columns)
+  double* cb_rec;         // kPsRecDoubles per CTA of pass 2 (kPsThreads columns): {n2, S, largest
+                          // per-column ratio, its column} -- the last two in the coordinate-wise form
   unsigned int* tickets;  // one counter, zero at entry and again on return
   double* stats;          // header + one shard record
   int64_t* b_next;
@@ -268,10 +269,42 @@ __global__ void __launch_bounds__(kPsThreads, kPsCtasPerSM)
 // Pass 2 and the decision (see the top of the file).
 constexpr int kPsTicketDoubles = 2;    // room for the ticket counter in stats_out (keeps 16-byte alignment)
 constexpr int kPsMergeInFlight = 16;  // row blocks of a column in flight at once
+constexpr int kPsRecDoubles = 4;      // doubles per record of a merge CTA
 
+// The running maximum of {ratio, column} with ties to the lower column; a NaN ratio never wins.
+__device__ __forceinline__ void ps_take_max(double& r, double& idx, double r2, double idx2) {
+  if (r2 > r || (r2 == r && idx2 < idx)) {
+    r = r2;
+    idx = idx2;
+  }
+}
+__device__ __forceinline__ void ps_block_max(double& r, double& idx, double* sm /* 2 per warp */) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const double r2 = __shfl_down_sync(0xffffffffu, r, off);
+    const double i2 = __shfl_down_sync(0xffffffffu, idx, off);
+    ps_take_max(r, idx, r2, i2);
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) {
+    sm[2 * warp] = r;
+    sm[2 * warp + 1] = idx;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0)
+    for (int w = 1; w < kPsThreads / 32; ++w) ps_take_max(r, idx, sm[2 * w], sm[2 * w + 1]);
+  __syncthreads();
+}
+
+// CW: the coordinate-wise test in its per-sample form (Sec. 4, Proposition 1, with the sample
+// variance of the Var definition before Eq. 3): per column i the ratio M2_i / gbar_i^2 (zero when
+// M2_i = 0, +inf when only gbar_i = 0), the decision from the largest one,
+// T = (max_i ratio_i / (b-1)) / eta^2, and the column where it occurs.
+template <bool CW>
 __global__ void __launch_bounds__(kPsThreads)
     persample_merge_kernel(const __grid_constant__ PersampleParams prm) {
   __shared__ double red[(kPsThreads / 32) * 3];
+  __shared__ double red_max[(kPsThreads / 32) * 2];
   __shared__ int s_last;
   const int tid = threadIdx.x;
   const int64_t c = static_cast<int64_t>(blockIdx.x) * kPsThreads + tid;
@@ -281,6 +314,7 @@ __global__ void __launch_bounds__(kPsThreads)
   const double inv_full = 1.0 / n_full, inv_last = 1.0 / static_cast<double>(n_last);
   grid_dependency_wait();
   double a = 0.0, sdev = 0.0, unused = 0.0;
+  double rmax = -1.0, rarg = static_cast<double>(c);  // -1: no column (or only NaN ratios) yet
   if (c < prm.d) {
     double su[kPsMergeInFlight], mm[kPsMergeInFlight];
     double tot = 0.0;
@@ -335,14 +369,24 @@ __global__ void __launch_bounds__(kPsThreads)
     prm.gbar[c] = gb;
     a = static_cast<double>(gb) * static_cast<double>(gb);
     sdev = m2;
+    if (CW) {
+      const double ratio = (m2 == 0.0) ? 0.0 : m2 / (mean * mean);
+      if (ratio > rmax) rmax = ratio;  // a NaN ratio leaves -1
+    }
   }
   block_reduce3<kPsThreads / 32>(a, sdev, unused, red);
+  if (CW) ps_block_max(rmax, rarg, red_max);
   // One fence per CTA: thread 0 wrote the record itself; its fence publishes it before the
   // ticket is drawn, and on the winning side it fences again before the barrier releases the
   // CTA to read the other records.
   if (tid == 0) {
-    __stcg(prm.cb_rec + 2 * static_cast<int64_t>(blockIdx.x), a);
-    __stcg(prm.cb_rec + 2 * static_cast<int64_t>(blockIdx.x) + 1, sdev);
+    double* rec = prm.cb_rec + kPsRecDoubles * static_cast<int64_t>(blockIdx.x);
+    __stcg(rec, a);
+    __stcg(rec + 1, sdev);
+    if (CW) {
+      __stcg(rec + 2, rmax);
+      __stcg(rec + 3, rarg);
+    }
     __threadfence();
     s_last = atomicAdd(prm.tickets, 1u) == gridDim.x - 1u;
     if (s_last) __threadfence();
@@ -352,16 +396,27 @@ __global__ void __launch_bounds__(kPsThreads)
 
   // records in index order: thread t takes t, t + 128, ...; then the fixed tree
   double n2 = 0.0, S = 0.0;
+  rmax = -1.0;
+  rarg = 0.0;
   for (int64_t cb = tid; cb < static_cast<int64_t>(gridDim.x); cb += kPsThreads) {
-    n2 += __ldcg(prm.cb_rec + 2 * cb);
-    S += __ldcg(prm.cb_rec + 2 * cb + 1);
+    const double* rec = prm.cb_rec + kPsRecDoubles * cb;
+    n2 += __ldcg(rec);
+    S += __ldcg(rec + 1);
+    if (CW) ps_take_max(rmax, rarg, __ldcg(rec + 2), __ldcg(rec + 3));
   }
   block_reduce3<kPsThreads / 32>(n2, S, unused, red);
+  if (CW) ps_block_max(rmax, rarg, red_max);
   if (tid == 0) {
     const double norm = static_cast<double>(prm.b - 1);
     double T;
     int flags;
-    const int64_t b_next = decide_device(S, n2, norm, prm.eta, prm.b, &T, &flags);
+    if (CW && rmax < 0.0) {  // every ratio was NaN: the sums are non-finite and say so
+      rmax = 0.0;
+      rarg = 0.0;
+    }
+    const int64_t b_next =
+        CW ? decide_coordwise_device(S, n2, rmax, norm, prm.eta, prm.b, &T, &flags)
+           : decide_device(S, n2, norm, prm.eta, prm.b, &T, &flags);
     const double nan = __longlong_as_double(0x7ff8000000000000ll);
     prm.stats[ABS_STAT_N2] = n2;
     prm.stats[ABS_STAT_S] = S;
@@ -370,12 +425,12 @@ __global__ void __launch_bounds__(kPsThreads)
     prm.stats[ABS_STAT_FLAGS] = static_cast<double>(flags);
     prm.stats[ABS_STAT_NORM] = norm;
     prm.stats[ABS_STAT_NCHUNKS] = static_cast<double>(gridDim.x);
-    prm.stats[ABS_STAT_ARGMAX] = 0.0;
+    prm.stats[ABS_STAT_ARGMAX] = CW ? rarg : 0.0;
     double* rec = prm.stats + ABS_STATS_HEADER;  // the one shard record
     rec[0] = n2;
     rec[1] = S;
-    rec[2] = nan;
-    rec[3] = 0.0;
+    rec[2] = CW ? rarg : nan;
+    rec[3] = CW ? T : 0.0;
     *prm.b_next = b_next;
     *prm.tickets = 0u;  // ready for the next call
   }

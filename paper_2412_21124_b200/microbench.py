@@ -113,7 +113,8 @@ def run_point(call, d, K, dtype, n_shards=1, steps=None, warmup=3, gbar=False, b
                                              None, s["b_next"], s["p"], s["m"], s["v"], HP,
                                              100 + i, shard_offsets=offs)
         else:
-            B.abs_persample_norm_test(s["G"], 0.1, s["stats"], s["gbar"], s["b_next"])
+            fn = B.abs_persample_norm_test_coordwise if coordwise else B.abs_persample_norm_test
+            fn(s["G"], 0.1, s["stats"], s["gbar"], s["b_next"])
 
     for i in range(warmup):
         one(i)
@@ -192,7 +193,8 @@ REPORT_POINTS = (
        ("adamw", GPT2, 0, "f32", 1, {"mixed": True})]
     + [("persample", 16_384, 0, "f32", 1, {"b": b}) for b in (4096, 1024, 256, 32)]
     + [("persample", 65_536, 0, "f32", 1, {"b": 4096}), ("persample", 16_384, 0, "bf16", 1, {"b": 4096}),
-       ("persample", 65_536, 0, "bf16", 1, {"b": 8192})]
+       ("persample", 65_536, 0, "bf16", 1, {"b": 8192}),
+       ("persample", 16_384, 0, "f32", 1, {"b": 4096, "coordwise": True})]
     + [("fused", GPT2, 8, "bf16", 1, {"gbar": True}), ("fused", GPT2, 8, "bf16", 1, {"mixed": True}),
        ("fused", 1_048_576, 4, "f32", 1, {})]
     + [("fused", GPT2, K, "bf16", 1, {}) for K in (6, 12, 20, 24, 27, 31, 36, 40, 44, 48, 52, 56,

@@ -419,6 +419,7 @@ def test_adamw_rejects_pointers(L):
 ])
 def test_persample_rejects(L, args, status):
     assert L.abs_persample_norm_test(*args) == status
+    assert L.abs_persample_norm_test_coordwise(*args) == status
 
 
 # ---- aliasing: outputs may not overlap the gradients or each other ------------------------

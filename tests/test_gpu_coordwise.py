@@ -255,3 +255,118 @@ def test_coordwise_config2_full_size():
     torch.cuda.synchronize()
     assert torch.equal(p, q) and torch.equal(m, mq) and torch.equal(v, vq)
     assert torch.equal(stats[:2], stats2[:2])
+
+
+# ------------------------------------------------------------- per-sample form
+def persample_cw_check(G, eta, rel=1e-5):
+    """abs_persample_norm_test_coordwise against the oracle's per-sample coordinate-wise test."""
+    b, d = G.shape
+    stats = absnt.alloc_persample_stats(b, d, DEV)
+    gbar = torch.full((d,), -3.0, dtype=torch.float32, device=DEV)
+    b_next = torch.full((1,), -7, dtype=torch.int64, device=DEV)
+    absnt.abs_persample_norm_test_coordwise(G, eta, stats, gbar, b_next)
+    torch.cuda.synchronize()
+    got = absnt.read_stats(stats)
+    host = to_host(G) if G.dtype == torch.bfloat16 else G.cpu().numpy()
+    ref = orc.persample_coordwise(host, eta, want_ratios=True)
+    assert got["norm"] == b - 1 and math.isnan(got["Q"])
+    if math.isfinite(ref["n2"]) and math.isfinite(ref["S"]):
+        assert_sum_close(got["n2"], ref["n2"], "n2")
+        if ref["S"] == 0.0:
+            assert got["S"] == 0.0
+        else:
+            assert_sum_close(got["S"], ref["S"], "S")
+        assert_vec_close(gbar, ref["gbar"], "gbar")
+    assert got["flags"] == ref["flags"], (got, ref["flags"])
+    if math.isnan(ref["T"]):
+        assert math.isnan(got["T"])
+    else:
+        assert close_or_both_inf(got["T"], ref["T"], rel), (got["T"], ref["T"])
+        i = got["argmax"]
+        assert 0 <= i < d
+        if math.isinf(ref["T"]):
+            assert math.isinf(ref["ratios"][i])
+        else:
+            assert ref["ratios"][i] >= (1.0 - rel) * ref["T"]
+        assert got["shards"][0][2] == i and got["shard_max"][0] == got["T"]
+    if margin_ok(ref["T"], b):
+        assert int(b_next.item()) == ref["b_next"]
+    return got, ref, int(b_next.item())
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("b,d,ld,shift", [(2, 5, 5, 0), (33, 300, 320, 0), (100, 2051, 2052, 1),
+                                          (257, 4096, 4096, 0), (1000, 777, 780, 0),
+                                          (2049, 515, 516, 0), (65, 40_000, 40_000, 0)])
+def test_persample_coordwise_shapes(b, d, ld, shift, dtype):
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(b * 139 + d)
+    buf = torch.empty(b * ld + shift, dtype=torch.float32, device=DEV)
+    buf.normal_(generator=gen)
+    buf.mul_(0.3).add_(0.2)
+    G = buf.to(dtype)[shift:].view(b, ld)[:, :d]
+    persample_cw_check(G, 0.3)
+
+
+def test_persample_coordwise_disagrees_with_the_summed_test():
+    """One column with a mean close to zero dominates the coordinate-wise statistic while the
+    summed test (Eq. 3) still passes: the two calls decide differently on the same matrix."""
+    b, d = 64, 3000
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(3)
+    G = torch.empty(b, d, device=DEV).normal_(generator=gen).mul_(0.05).add_(1.0)
+    G[:, 1234] -= G[:, 1234].mean() - 1e-4    # this column's mean is 1e-4, its spread stays
+    eta = 0.5
+    got, ref, b_cw = persample_cw_check(G, eta)
+    assert got["argmax"] == 1234 and b_cw > b
+    stats = absnt.alloc_persample_stats(b, d, DEV)
+    gbar = torch.empty(d, dtype=torch.float32, device=DEV)
+    b_next = torch.zeros(1, dtype=torch.int64, device=DEV)
+    absnt.abs_persample_norm_test(G, eta, stats, gbar, b_next)
+    torch.cuda.synchronize()
+    assert int(b_next.item()) == b    # the summed test keeps the batch size
+
+
+def test_persample_coordwise_zero_rules_ties_and_nonfinite():
+    b, d = 40, 700
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(4)
+    base = torch.empty(b, d, device=DEV).normal_(generator=gen).mul_(0.1).add_(0.5)
+    # a column of identical values has T_i = 0, also when that value is zero
+    G = base.clone()
+    G[:, 10] = 0.25
+    G[:, 11] = 0.0
+    got, ref, _ = persample_cw_check(G, 0.3)
+    assert ref["ratios"][10] == 0.0 and ref["ratios"][11] == 0.0
+    # two identical columns tie: the lower index is reported
+    G = base.clone()
+    G[:, 5] = G[:, 600] = torch.linspace(-1.0, 1.001, b, device=DEV)
+    got, ref, _ = persample_cw_check(G, 0.3)
+    assert got["argmax"] == 5 == ref["argmax"]
+    # a column whose values cancel exactly: positive variance, zero mean -> +inf, DEGENERATE
+    G = base.clone()
+    half = torch.linspace(0.1, 1.0, b // 2, device=DEV)
+    G[:, 77] = torch.cat([half, -half])
+    got, ref, b_next = persample_cw_check(G, 0.3)
+    assert got["T"] == math.inf and got["argmax"] == 77 and b_next == INT64_MAX
+    assert got["flags"] == absnt.ABS_FLAG_DEGENERATE | absnt.ABS_FLAG_VIOLATED
+    # a NaN anywhere: NONFINITE, the batch size stays
+    G = base.clone()
+    G[17, 300] = float("nan")
+    got, ref, b_next = persample_cw_check(G, 0.3)
+    assert got["flags"] & absnt.ABS_FLAG_NONFINITE and b_next == b
+
+
+def test_persample_coordwise_hand_cases():
+    """Hand cases H8 and H9 with their rows as the samples (b = 2, normalisation b - 1 = 1)."""
+    cases = json.load(open(GOLDEN))["coordwise"]
+    c = cases[0]
+    G = torch.tensor(c["grads"], dtype=torch.float32, device=DEV)
+    got, ref, b_next = persample_cw_check(G, c["eta"])
+    assert got["T"] == c["T_persample"] and got["argmax"] == c["argmax"]
+    assert b_next == c["b_next_persample"]
+    c = cases[1]
+    G = torch.tensor(c["grads"], dtype=torch.float32, device=DEV)
+    got, ref, b_next = persample_cw_check(G, c["eta"])
+    assert got["T"] == math.inf and got["argmax"] == c["argmax"] and got["flags"] == c["flags"]
+    assert b_next == INT64_MAX
