@@ -79,6 +79,13 @@ struct FinalizeParams {
 __device__ __forceinline__ void grid_dependency_wait() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
+// Lets the next kernel of the stream be scheduled (it was launched with the same attribute)
+// once every CTA of this grid has executed this or exited.  The dependent still waits at its
+// own grid_dependency_wait for this grid's completion, so only its launch latency and the work
+// it does before that wait move forward.
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 // ---- streaming memory access --------------------------------------------------------
 // Gradients are read exactly once and never written: non-coherent path, no L1 allocation.

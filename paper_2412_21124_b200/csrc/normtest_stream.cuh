@@ -919,6 +919,11 @@ __global__ void __launch_bounds__(kFinalizeThreads)
   // The barrier touches no global memory, so it sits before the dependency wait and overlaps
   // the tail of the preceding kernel.
   cluster.sync();
+  // This kernel occupies at most eight SMs: the next kernel of the stream (with the library's
+  // calls back to back, the next call's streaming kernel) may be scheduled now and run up to its
+  // own dependency wait -- which still holds it until this grid has completed -- so its launch and
+  // prologue are off the critical path (0.5-0.6 us per call: d = 1M 10.4 -> 9.8 us).
+  grid_launch_dependents();
   grid_dependency_wait();
   for (int i = rank * kFinalizeWarps + warp; i < n_slices; i += n_warps) {
     // the shard of slice i: the last s with slice_prefix[s] <= i

@@ -312,6 +312,9 @@ __global__ void __launch_bounds__(kPsThreads)
   const int64_t n_last = prm.b - static_cast<int64_t>(nrb - 1) * prm.rows_per_block;
   const double n_full = static_cast<double>(prm.rows_per_block);
   const double inv_full = 1.0 / n_full, inv_last = 1.0 / static_cast<double>(n_last);
+  // a small grid: the next kernel of the stream may be scheduled and run up to its own
+  // dependency wait (b = 4096, d = 16384: 46.8 -> 46.4 us per call; b = 256: 10.9 -> 11.1)
+  grid_launch_dependents();
   grid_dependency_wait();
   double a = 0.0, sdev = 0.0, unused = 0.0;
   double rmax = -1.0, rarg = static_cast<double>(c);  // -1: no column (or only NaN ratios) yet
