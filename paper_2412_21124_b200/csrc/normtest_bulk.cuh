@@ -7,7 +7,8 @@
 // stage and arms the stage's mbarrier with the byte count; all 256 threads wait on that
 // mbarrier, take 4 coordinates each from shared memory, do the per-coordinate math in
 // registers, write p, m, v (and gbar) back into the stage, and the elected thread sends them
-// to global memory with bulk stores.  kBulkStages stages keep the next tiles' loads in
+// to global memory with bulk stores (the test alone, which writes only gbar, stores it straight
+// from registers and keeps nothing but gradients in its stages).  kBulkStages stages keep the next tiles' loads in
 // flight while a tile is computed.  Measured on the K=8 bf16 fused step this request pattern
 // sustains about 2.5% more bandwidth than 128-bit loads issued per thread (the copy engine
 // issues large, aligned requests and the SM spends no load/store instructions on them).
@@ -33,7 +34,8 @@ constexpr int kSmemPerSM = 224 * 1024;   // budget for dynamic shared memory per
 // bytes of one stage of `tile` coordinates
 template <typename GT, int KB, bool ADAM>
 __host__ __device__ constexpr int bulk_stage_bytes(int tile) {
-  return tile * (KB * static_cast<int>(sizeof(typename GT::scalar)) + (ADAM ? 12 : 0) + 4);
+  // fused: the K gradient segments, p, m, v and gbar; the test alone: the gradients only
+  return tile * (KB * static_cast<int>(sizeof(typename GT::scalar)) + (ADAM ? 16 : 0));
 }
 // Shape of the staged kernel for one (dtype, K, fused) combination: coordinates per stage
 // (4 per thread), stages per CTA, CTAs per SM.  tile == 0: not offered.  Measured and
@@ -45,7 +47,7 @@ struct BulkShape {
 template <typename GT, int KB, bool ADAM>
 __host__ __device__ constexpr BulkShape bulk_shape() {
   // The test alone has small stages (no optimizer state), so three CTAs of three or more
-  // stages fit for up to 10 bf16 / 5 fp32 workers: 24 warps per SM instead of 16 cover the
+  // stages fit for up to 12 bf16 / 6 fp32 workers: 24 warps per SM instead of 16 cover the
   // per-tile barrier and the wait for a tile's arrival better (bf16 K=7 6.64 -> 6.91 TB/s, K=8
   // 6.70 -> 6.88, K=9, 10 +3%; fp32 K=3 6.65 -> 6.91; K=8 bf16 on 1.24G coordinates in 8 shards
   // 6.88 -> 7.11; bf16 K=6, which used to prefer the register-direct kernel, 6.64 -> 6.95; nothing
@@ -163,7 +165,7 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
   constexpr int FB = kBulkTile * 4;                                              // fp32 segment
   constexpr int OFF_P = KB * GB, OFF_M = OFF_P + (ADAM ? FB : 0), OFF_V = OFF_M + (ADAM ? FB : 0);
   constexpr int OFF_GBAR = OFF_V + (ADAM ? FB : 0);
-  constexpr int STAGE = OFF_GBAR + FB;
+  constexpr int STAGE = OFF_GBAR + (ADAM ? FB : 0);
   static_assert(STAGE == bulk_stage_bytes<GT, KB, ADAM>(TILE), "stage layout");
   extern __shared__ __align__(128) unsigned char stages[];
   __shared__ uint64_t full[kBulkStages];
@@ -276,7 +278,7 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
         acc_S += static_cast<double>(row_S);
         if (WITHQ) acc_Q += static_cast<double>(row_Q);
 
-        if (ADAM) {
+        if constexpr (ADAM) {
           *reinterpret_cast<float4*>(st + OFF_P + tid * 16) = pw;
           *reinterpret_cast<float4*>(st + OFF_M + tid * 16) = pm;
           *reinterpret_cast<float4*>(st + OFF_V + tid * 16) = pv;
@@ -284,21 +286,26 @@ __global__ void __launch_bounds__(TILE / 4, CTAS)
           // coordinate do not earn a stage segment
           if (prm.p16)
             st_bf16x4(prm.p16 + cg.lo + static_cast<int64_t>(i) * kBulkTile + tid * 4, pw);
-        }
-        if (prm.gbar)
-          *reinterpret_cast<float4*>(st + OFF_GBAR + tid * 16) =
-              make_float4(gb[0], gb[1], gb[2], gb[3]);
-        fence_generic_to_async_smem();
-        __syncthreads();  // tile consumed by everyone, results visible to the copy engine
-        if (tid == 0) {
-          const int64_t e = cg.lo + static_cast<int64_t>(i) * kBulkTile;
-          if (ADAM) {
+          if (prm.gbar)
+            *reinterpret_cast<float4*>(st + OFF_GBAR + tid * 16) =
+                make_float4(gb[0], gb[1], gb[2], gb[3]);
+          fence_generic_to_async_smem();
+          __syncthreads();  // tile consumed by everyone, results visible to the copy engine
+          if (tid == 0) {
+            const int64_t e = cg.lo + static_cast<int64_t>(i) * kBulkTile;
             bulk_store(prm.p + e, st + OFF_P, FB);
             bulk_store(prm.m + e, st + OFF_M, FB);
             bulk_store(prm.v + e, st + OFF_V, FB);
+            if (prm.gbar) bulk_store(prm.gbar + e, st + OFF_GBAR, FB);
+            bulk_commit();
           }
-          if (prm.gbar) bulk_store(prm.gbar + e, st + OFF_GBAR, FB);
-          bulk_commit();
+        } else {
+          // the test alone writes only gbar (4 of K*s + 4 bytes per coordinate): straight from
+          // registers, so that the stage holds nothing but gradients (smaller stages: more of
+          // them, or a third CTA, fit) -- +0.5% at bf16 K=8 by itself
+          st_stream_16(prm.gbar + cg.lo + static_cast<int64_t>(i) * kBulkTile + tid * 4,
+                       make_float4(gb[0], gb[1], gb[2], gb[3]));
+          __syncthreads();  // tile consumed by everyone: its stage may be refilled
         }
       }
       tiles_done += static_cast<uint32_t>(n_tiles);
