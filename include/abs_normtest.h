@@ -12,7 +12,9 @@
  *
  * Conventions that hold for every launching entry point
  *   - "device" pointers are memory of the CUDA device that is current on the calling
- *     thread; "host" pointers are ordinary memory read during the call only.
+ *     thread ("grads" buffers, which are only read, may also be memory of a peer device that
+ *     the current one can address); "host" pointers are ordinary memory read during the
+ *     call only.
  *   - The caller owns every buffer.  The library allocates no device memory and
  *     keeps no state between calls that a result depends on (what it does keep, on the
  *     host: abs_last_cuda_error, and which kernel attributes it has set on which device).
