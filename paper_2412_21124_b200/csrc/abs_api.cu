@@ -471,26 +471,31 @@ int run_accumulate(const void* const* grads, int K, int64_t d, abs_dtype dtype,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid(static_cast<unsigned>(L.n_chunks)), block(kThreads);
   cudaError_t e;
-  // few gradients per call: several thread-rows in flight per thread, 128 bytes of gradients
-  // either way (fp32: 16-byte vectors, bf16: 8-byte vectors; eight rows fit for a single bf16
-  // gradient and spill otherwise).  With AdamW the state vectors are in flight as
+  // up to one group of gradients per call (16 bf16 / 8 fp32): several thread-rows in flight per
+  // thread, 128 bytes of gradients or more either way (fp32: 16-byte vectors, bf16: 8-byte
+  // vectors; eight rows fit for a single bf16 gradient and spill otherwise; two rows of a whole
+  // group at two CTAs per SM: bf16 K=9 4.81 -> 5.77 TB/s, K=12 5.20 -> 6.22, fp32 K=5 5.15 -> 6.21).  With AdamW the state vectors are in flight as
   // well: two rows up to four gradients, one beyond.
   if (fused) {
     if (dtype == ABS_F32)
-      e = K <= 4 ? launch_pdl(normtest_accumulate_kernel<F32, 2, 4, true>, grid, block, st, prm, cy)
-                 : launch_pdl(normtest_accumulate_kernel<F32, 1, 1, true>, grid, block, st, prm, cy);
+      e = K <= 4   ? launch_pdl(normtest_accumulate_kernel<F32, 2, 4, true>, grid, block, st, prm, cy)
+          : K <= 8 ? launch_pdl(normtest_accumulate_kernel<F32, 1, 8, true>, grid, block, st, prm, cy)
+                   : launch_pdl(normtest_accumulate_kernel<F32, 1, 1, true>, grid, block, st, prm, cy);
     else
-      e = K <= 4   ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 4, true>, grid, block, st, prm, cy)
-          : K <= 8 ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 8, true>, grid, block, st, prm, cy)
-                   : launch_pdl(normtest_accumulate_kernel<BF16H, 1, 1, true>, grid, block, st, prm, cy);
+      e = K <= 4    ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 4, true>, grid, block, st, prm, cy)
+          : K <= 8  ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 8, true>, grid, block, st, prm, cy)
+          : K <= 16 ? launch_pdl(normtest_accumulate_kernel<BF16H, 1, 16, true>, grid, block, st, prm, cy)
+                    : launch_pdl(normtest_accumulate_kernel<BF16H, 1, 1, true>, grid, block, st, prm, cy);
   } else if (dtype == ABS_F32) {
     e = K <= 2   ? launch_pdl(normtest_accumulate_kernel<F32, 4, 2, false>, grid, block, st, prm, cy)
         : K <= 4 ? launch_pdl(normtest_accumulate_kernel<F32, 2, 4, false>, grid, block, st, prm, cy)
+        : K <= 8 ? launch_pdl(normtest_accumulate_kernel<F32, 2, 8, false>, grid, block, st, prm, cy)
                  : launch_pdl(normtest_accumulate_kernel<F32, 1, 1, false>, grid, block, st, prm, cy);
   } else {
     e = K == 1   ? launch_pdl(normtest_accumulate_kernel<BF16H, 8, 1, false>, grid, block, st, prm, cy)
         : K <= 4 ? launch_pdl(normtest_accumulate_kernel<BF16H, 4, 4, false>, grid, block, st, prm, cy)
         : K <= 8 ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 8, false>, grid, block, st, prm, cy)
+        : K <= 16 ? launch_pdl(normtest_accumulate_kernel<BF16H, 2, 16, false>, grid, block, st, prm, cy)
                  : launch_pdl(normtest_accumulate_kernel<BF16H, 1, 1, false>, grid, block, st, prm, cy);
   }
   if (e != cudaSuccess) return cuda_fail(e);

@@ -133,12 +133,14 @@ __device__ __noinline__ void accumulate_scalar_row(const StreamParams& prm, cons
   sums[1] = row_S;
 }
 
+// KR > 1: the call has at most KR workers, whose loads are issued as one predicated batch.
 // ROWS > 1: calls with at most KR workers load ROWS thread-rows (ROWS * K gradient vectors and the
 // ROWS mean vectors: 128 bytes of gradients per thread for ROWS * KR = 8 vectors of 16 bytes or
 // 16 of 8 bytes) before the first is consumed; rows are consumed in order, so the sums have the
 // shape of the ROWS = 1 kernel and both give the same bits.
 template <typename GT, int ROWS, int KR, bool ADAM>
-__global__ void __launch_bounds__(kThreads, ADAM ? 2 : 3)
+__global__ void __launch_bounds__(
+    kThreads, (ADAM || ROWS * KR * static_cast<int>(sizeof(typename GT::raw_t)) > 128) ? 2 : 3)
     normtest_accumulate_kernel(const __grid_constant__ StreamParams prm,
                                const __grid_constant__ AccumCarry cy) {
   static_assert(GT::kVec == 4, "four coordinates per thread-row");
@@ -235,38 +237,51 @@ __global__ void __launch_bounds__(kThreads, ADAM ? 2 : 3)
       bool need_centre = !carry;  // uniform across the CTA
       if (carry) acc.init(ld_state_16(cy.mean_in + base));
       State st = load_state(base);  // in flight while the gradients are consumed
-      // N consecutive workers from k0: all loads first, then the arithmetic
-      auto piece = [&](int k0, auto n_tag) {
-        constexpr int N = decltype(n_tag)::value;
-        typename GT::raw_t raw[N];
+      if constexpr (KR > 1) {
+        // at most KR workers (the caller's promise for KR > 1): one predicated batch
+        typename GT::raw_t raw[KR];
 #pragma unroll
-        for (int k = 0; k < N; ++k) raw[k] = GT::load_vec(vec_ptr(k0 + k, base));
-        if (need_centre) {
-          acc.init_from(raw[0]);
-          need_centre = false;
-        }
+        for (int k = 0; k < KR; ++k)
+          if (k < K) raw[k] = GT::load_vec(vec_ptr(k, base));
+        if (need_centre) acc.init_from(raw[0]);
 #pragma unroll
-        for (int k = 0; k < N; ++k) acc.add(raw[k]);
-      };
-      int k0 = 0;
+        for (int k = 0; k < KR; ++k)
+          if (k < K) acc.add(raw[k]);
+      } else {
+        // N consecutive workers from k0: all loads first, then the arithmetic
+        auto piece = [&](int k0, auto n_tag) {
+          constexpr int N = decltype(n_tag)::value;
+          typename GT::raw_t raw[N];
+#pragma unroll
+          for (int k = 0; k < N; ++k) raw[k] = GT::load_vec(vec_ptr(k0 + k, base));
+          if (need_centre) {
+            acc.init_from(raw[0]);
+            need_centre = false;
+          }
+#pragma unroll
+          for (int k = 0; k < N; ++k) acc.add(raw[k]);
+        };
+        // whole groups of H workers, then the rest in unpredicated pieces of 8, 4, 2, 1
+        int k0 = 0;
 #pragma unroll 1
-      for (; k0 + H <= K; k0 += H) {
-        piece(k0, std::integral_constant<int, H>{});
-        acc.close_group();
+        for (; k0 + H <= K; k0 += H) {
+          piece(k0, std::integral_constant<int, H>{});
+          acc.close_group();
+        }
+        if (H > 8 && ((K - k0) & 8)) {
+          piece(k0, std::integral_constant<int, 8>{});
+          k0 += 8;
+        }
+        if ((K - k0) & 4) {
+          piece(k0, std::integral_constant<int, 4>{});
+          k0 += 4;
+        }
+        if ((K - k0) & 2) {
+          piece(k0, std::integral_constant<int, 2>{});
+          k0 += 2;
+        }
+        if ((K - k0) & 1) piece(k0, std::integral_constant<int, 1>{});
       }
-      if (H > 8 && ((K - k0) & 8)) {
-        piece(k0, std::integral_constant<int, 8>{});
-        k0 += 8;
-      }
-      if ((K - k0) & 4) {
-        piece(k0, std::integral_constant<int, 4>{});
-        k0 += 4;
-      }
-      if ((K - k0) & 2) {
-        piece(k0, std::integral_constant<int, 2>{});
-        k0 += 2;
-      }
-      if ((K - k0) & 1) piece(k0, std::integral_constant<int, 1>{});
       acc.close_group();  // adds exact zeros when K is a multiple of H
       finish_row(acc, base, st);
     } else if (base < hi) {
