@@ -97,6 +97,7 @@ SPLITS = [
     [16, 17],                  # a whole group of 16 (bf16) / two of 8 (fp32) and a remainder
     [64, 36],                  # the largest call
     [1, 2, 4, 8, 16, 2],
+    [12, 9, 6, 15],            # part of a group: the predicated batch of the two-row kernels
 ]
 
 
@@ -239,7 +240,8 @@ def test_accumulate_config2_size_sampled():
 
 # ------------------------------------------------------------- closing call fused with AdamW
 CLOSING = [([8], "whole step"), ([7, 1], "one"), ([4, 4], "two rows"), ([3, 9], "general"),
-           ([1] * 5, "micro-batches"), ([20, 33], "groups")]
+           ([1] * 5, "micro-batches"), ([20, 33], "groups"), ([2, 6], "batch of six"),
+           ([3, 13], "batch of thirteen")]
 
 
 @pytest.mark.parametrize("inplace", [True, False], ids=["mean in place", "mean not written"])
