@@ -207,8 +207,8 @@ REPORT_POINTS = (
        ("fused", GPT2, 4, "f32", 1, {"coordwise": True}),
        ("fused", GPT2, 32, "bf16", 1, {"coordwise": True})]
     # the carry-in form: K new gradients merged into the running mean per call
-    + [("accumulate", GPT2, K, dt, 1, {}) for K in (1, 2, 4, 8, 16) for dt in ("bf16", "f32")]
-    + [("accumulate_adamw", GPT2, K, "bf16", 1, {}) for K in (1, 4, 8)]
+    + [("accumulate", GPT2, K, dt, 1, {}) for K in (1, 2, 4, 8, 9, 12, 16, 32) for dt in ("bf16", "f32")]
+    + [("accumulate_adamw", GPT2, K, "bf16", 1, {}) for K in (1, 4, 8, 16)]
     # the paper's own model sizes (Table 4), J = 4 workers, bf16
     + [("fused", d, 4, "bf16", 1, {}) for d in (304_600_000, 1_100_000_000, 3_400_000_000)])
 
