@@ -20,7 +20,8 @@
 // The chunk records have the layout of the other streaming kernels and go through the same
 // finalize kernel; the carry enters as one more addend: the CTA of a shard's first chunk adds
 // the shard's previous sum to its own partial.  Few workers per call leave little in flight,
-// so for m <= 4 a thread loads several thread-rows before it consumes the first.
+// so up to one group of workers (16 bf16 / 8 fp32) a thread loads several thread-rows, or two
+// rows of the whole group, before it consumes the first (the kernel's ROWS and KR).
 #pragma once
 #include "normtest_stream.cuh"
 
